@@ -1,0 +1,183 @@
+/*
+ * rosaq.h -- C ABI of the B200 (sm_100a) implementation of the ROSAQ inference
+ * hot path: the fused mixed-precision rotated linear  y = (x R) W',  W' = R^T W,
+ * with W' stored as one FP16 salient group plus INT4/INT3 groups of 128 input
+ * channels (fp16 scale and zero-point per group and output column).
+ *
+ * Notation follows the paper: X calibration activations [N][d], R rotation
+ * (eigenvectors of X^T X sorted by descending eigenvalue), W weight [d][d'],
+ * K salient channels.  (The paper writes Q(.) for the quantizer; here the
+ * quantizer is always spelled "quantize".)
+ *
+ * Conventions for every call
+ *   - All matrices are row-major.  Unless a parameter is marked HOST, pointers are
+ *     DEVICE pointers on the device the context was created for, and stay owned
+ *     by the caller; the library never frees or keeps them past the call's
+ *     completion on `stream` (exception: none).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls are asynchronous on it unless stated otherwise.
+ *   - Return value: ROSAQ_OK (0) or a negative rosaq_status.  Nothing is thrown,
+ *     printed or aborted.  Argument errors are detected before any launch.
+ *   - Device-side waits are bounded; if one expires the kernel records
+ *     ROSAQ_ERR_TIMEOUT in the context's device status word (read it with
+ *     rosaq_last_status) and returns, leaving the CUDA context usable.
+ *   - Handles (rosaq_ctx, rosaq_weight, rosaq_rotation) are owned by the library
+ *     and released with the matching *_destroy / *_free.  They are not
+ *     thread-safe; use one context per host thread and device.
+ */
+#ifndef ROSAQ_H_
+#define ROSAQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ROSAQ_OK = 0,
+  ROSAQ_ERR_INVALID_ARG = -1,       /* null pointer, non-positive size, bad enum */
+  ROSAQ_ERR_UNSUPPORTED_SHAPE = -2, /* size not a multiple of what the layout needs */
+  ROSAQ_ERR_ALIGNMENT = -3,         /* pointer or leading dimension not 16-byte aligned */
+  ROSAQ_ERR_ALLOC = -4,             /* device or host allocation failed */
+  ROSAQ_ERR_CUDA = -5,              /* a CUDA runtime/driver call failed */
+  ROSAQ_ERR_TIMEOUT = -6,           /* a bounded device-side wait expired */
+  ROSAQ_ERR_UNSUPPORTED_ARCH = -7   /* device is not compute capability 10.x */
+} rosaq_status;
+
+typedef enum { ROSAQ_F16 = 0, ROSAQ_F32 = 1 } rosaq_dtype;
+
+typedef struct rosaq_ctx rosaq_ctx;           /* per device: workspace + device status word */
+typedef struct rosaq_weight rosaq_weight;     /* one quantized linear in the kernels' tiled layout */
+typedef struct rosaq_rotation rosaq_rotation; /* one rotation R prepared for online use */
+
+/*
+ * Description of a rotation R (Section 3.1, Eq. 4; head-wise: Section 3.1.1, Eq. 6).
+ * R = blockdiag(q[0], ..., q[n_blocks-1]) followed by a column permutation:
+ * column j of R is column perm[j] of the block-diagonal matrix (perm NULL =
+ * identity).  n_blocks = 1 is the layer-wise dense rotation.  Columns are
+ * expected in descending-eigenvalue order, so that the first K are the salient
+ * ones (Section 3.2); the library does not check orthogonality.
+ */
+typedef struct {
+  int32_t d;           /* total dimension */
+  int32_t n_blocks;    /* d % n_blocks == 0 */
+  const void *q;       /* DEVICE [n_blocks][d/n_blocks][d/n_blocks] */
+  int32_t q_dtype;     /* ROSAQ_F32 for rosaq_quantize, ROSAQ_F16 for rosaq_rotation_create */
+  const int32_t *perm; /* DEVICE [d] or NULL; must be a permutation of 0..d-1 */
+} rosaq_rot;
+
+/* ---- context ---------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (must be compute capability 10.x, else
+ * ROSAQ_ERR_UNSUPPORTED_ARCH).  Allocates a small device status word and, lazily,
+ * a workspace for the rotated activations.  Synchronous. */
+int rosaq_create(rosaq_ctx **out, int device);
+int rosaq_destroy(rosaq_ctx *ctx);
+
+/* Static, never-NULL description of a status code. */
+const char *rosaq_strerror(int status);
+
+/* Synchronizes `stream`, then returns and clears the device status word
+ * (ROSAQ_OK or ROSAQ_ERR_TIMEOUT), or ROSAQ_ERR_CUDA if the stream reports an error. */
+int rosaq_last_status(rosaq_ctx *ctx, void *stream);
+
+/* Test hook: upper bound, in polling iterations, of every device-side wait
+ * (default 1<<26; a positive value replaces it).  Returns the previous value. */
+int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
+
+/* Selects the rosaq_linear / rosaq_rotate implementation: 0 = tensor-core path
+ * (tcgen05 + TMEM; default), 1 = plain CUDA-core path (slow; for debugging and
+ * cross-checks -- it is still a GPU kernel of this library).  Returns the previous value. */
+int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl);
+
+/* ---- calibration: Eq. 4, left-hand side ---------------------------------------- */
+
+/*
+ * C += X^T X  (uncentred, unnormalised Gram matrix), fp32 accumulation.
+ *   X        [n_tokens][ldx] of x_dtype (ROSAQ_F16 or ROSAQ_F32); only the first d columns are read
+ *   n_blocks 1: C is [d][d].  H > 1 (head-wise, Section 3.1.1): C is [H][d/H][d/H], the
+ *            independent Gram matrices of the column slices [h d/H, (h+1) d/H)
+ *   C        fp32, zeroed by the caller before the first chunk; may be called
+ *            repeatedly to stream a calibration set through in chunks
+ * The full square is written (both triangles).  d % 8 == 0, (d / n_blocks) % 8 == 0, X 16-byte aligned.
+ */
+int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens, int d,
+                    int64_t ldx, int n_blocks, float *C, void *stream);
+
+/* ---- offline: rotate + quantize + pack (Eq. 3, Section 3.3) -------------------- */
+
+/*
+ * Builds the mixed-precision representation of W' = R^T W.
+ *   W         fp16 [d_in][d_out]
+ *   rot       R with q_dtype ROSAQ_F32, rot->d == d_in; NULL = identity (the paper's
+ *             rotation-less "Mixed" baseline)
+ *   bits      3 or 4;  group must be 128;  k_salient a multiple of 128 in [0, d_in]
+ * W' is accumulated in fp32 as one fused multiply-add per term, input channel
+ * ascending, so that its bits (and therefore every code) are reproducible.
+ * Rows [0, k_salient) of W' are rounded to fp16 and kept; every further group of
+ * 128 rows is quantized per output column with asymmetric min/max round-to-nearest:
+ *   s = fp16(max(hi-lo, 1e-5) / (2^bits-1)), z = clamp(-rint(lo/s), 0, 2^bits-1),
+ *   code = clamp(rint(w/s) + z, 0, 2^bits-1), all IEEE fp32, ties to even.
+ * Allocates the result (*out, release with rosaq_weight_free) and a temporary fp32
+ * W' of d_in*d_out floats that is freed before returning.  Synchronizes `stream`.
+ * d_in % 128 == 0 required; d_out >= 1 (padded internally to a multiple of 128).
+ */
+int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot,
+                   int bits, int group, int k_salient, rosaq_weight **out, void *stream);
+
+/*
+ * Interchange layout of a quantized weight (r = row index inside the non-salient part):
+ *   qw       uint32; INT4: [(d_in-K)/8][d_out], code of row r in bits [4(r%8), +4) of qw[r/8][n];
+ *            INT3: [(d_in-K)/32*3][d_out], rows in blocks of 32 forming the 96-bit little-endian
+ *            string qw[3(r/32)+0..2][n], code of row r in bits [3(r%32), +3)
+ *   scales, zeros   fp16 [(d_in-K)/128][d_out]
+ *   salient  fp16 [K][d_out]
+ * export writes the four arrays (any may be NULL to skip it); import builds a handle
+ * from them.  Both run on `stream`; import also allocates and synchronizes.
+ */
+int rosaq_weight_export(rosaq_ctx *ctx, const rosaq_weight *w, uint32_t *qw, void *scales_f16,
+                        void *zeros_f16, void *salient_f16, void *stream);
+int rosaq_weight_import(rosaq_ctx *ctx, int d_in, int d_out, int bits, int group, int k_salient,
+                        const uint32_t *qw, const void *scales_f16, const void *zeros_f16,
+                        const void *salient_f16, rosaq_weight **out, void *stream);
+int rosaq_weight_free(rosaq_weight *w);
+/* HOST out-parameters (any may be NULL); device_bytes = size of the tiled representation. */
+int rosaq_weight_info(const rosaq_weight *w, int *d_in, int *d_out, int *bits, int *group,
+                      int *k_salient, int64_t *device_bytes);
+
+/* ---- online: x R, and (x R) W' (Eq. 3; Eq. 6 for block-diagonal R) -------------- */
+
+/*
+ * Prepares R (q_dtype ROSAQ_F16) for the online rotation: re-tiles it for the
+ * kernels and inverts the permutation.  (d / n_blocks) % 128 == 0 required.
+ * Allocates; synchronizes `stream`.
+ */
+int rosaq_rotation_create(rosaq_ctx *ctx, const rosaq_rot *rot, rosaq_rotation **out, void *stream);
+int rosaq_rotation_free(rosaq_rotation *r);
+
+/*
+ * x_rot[M][ldxr] (fp16) = x[M][ldx] (fp16) . R, fp32 accumulation, rounded once to fp16.
+ * Linears that read the same activation (q/k/v, gate/up) share one rotation, so it
+ * is exposed on its own.  ldx, ldxr in elements, multiples of 8; 1 <= M.
+ */
+int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r,
+                 void *x_rot, int64_t ldxr, void *stream);
+
+/*
+ * y[M][ldy] (fp16) = (x[M][ldx] (fp16) . R) . W^,  where W^ is the dequantized
+ * mixed-precision weight: row i < K is the stored fp16 value, otherwise
+ * (code - zero) * scale rounded to fp16; fp32 accumulation; y rounded once to fp16.
+ *   r == NULL : x is already rotated (only the GEMM stage runs)
+ *   r != NULL : x . R goes through the context workspace (grown on demand: this call
+ *               may then allocate and synchronize once), then the GEMM stage runs
+ * Only the first d_out columns of each y row are written.  ldx, ldy multiples of 8.
+ */
+int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r,
+                 const rosaq_weight *w, void *y, int64_t ldy, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROSAQ_H_ */

@@ -308,7 +308,7 @@ void oracle_quantize(const float *Wp, int d_in, int n_cols, int bits, int group,
       if (sb == 0x7c00) sb = 0x7bff;
       float sf = (float)f16_bits_to_double(sb);
       float z = -rintf(lo / sf);
-      if (z < 0.0f) z = 0.0f;
+      if (z <= 0.0f) z = 0.0f; /* also turns -0 (lo == +0) into +0 */
       if (z > qmax) z = qmax;
       scales[(int64_t)g * n_cols + n] = sb;
       zeros[(int64_t)g * n_cols + n] = f32_to_f16_bits(z); /* small integer: exact */

@@ -1,0 +1,378 @@
+// extern "C" entry points of librosaq: argument checks, handle management, dispatch.
+#include <new>
+
+#include "rosaq_internal.cuh"
+
+using namespace rosaq;
+
+namespace {
+
+int cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return ROSAQ_OK;
+  (void)cudaGetLastError();
+  return e == cudaErrorMemoryAllocation ? ROSAQ_ERR_ALLOC : ROSAQ_ERR_CUDA;
+}
+
+// Fills the geometry of a tiled operand; no allocation.
+TiledOperand make_geometry(int d_in, int d_out, int bits, int g_fp16, int g_quant, int block_groups) {
+  TiledOperand t{};
+  t.d_in = d_in;
+  t.d_out = d_out;
+  t.n_tiles = (d_out + kTileN - 1) / kTileN;
+  t.bits = bits;
+  t.g_fp16 = g_fp16;
+  t.g_quant = g_quant;
+  t.block_groups = block_groups;
+  t.tile_stride = (long long)g_fp16 * kFp16TileBytes + (long long)g_quant * quant_tile_bytes(bits);
+  t.bytes = t.tile_stride * t.n_tiles;
+  return t;
+}
+
+int alloc_blob(TiledOperand *t) {
+  void *p = nullptr;
+  size_t bytes = t->bytes > 0 ? (size_t)t->bytes : 16;
+  int st = cuda_status(cudaMalloc(&p, bytes));
+  if (st != ROSAQ_OK) return st;
+  t->blob = static_cast<uint8_t *>(p);
+  return ROSAQ_OK;
+}
+
+int check_quant_args(int d_in, int d_out, int bits, int group, int k_salient) {
+  if (d_in <= 0 || d_out <= 0) return ROSAQ_ERR_INVALID_ARG;
+  if (bits != 3 && bits != 4) return ROSAQ_ERR_INVALID_ARG;
+  if (group != kGroup) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (d_in % kGroup != 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (k_salient < 0 || k_salient > d_in || k_salient % kGroup != 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  return ROSAQ_OK;
+}
+
+int ensure_workspace(rosaq_ctx *ctx, size_t bytes, cudaStream_t s) {
+  if (ctx->ws_bytes >= bytes) return ROSAQ_OK;
+  // the old buffer may still be in use by work queued on some stream
+  int st = cuda_status(cudaDeviceSynchronize());
+  if (st != ROSAQ_OK) return st;
+  (void)s;
+  if (ctx->ws) (void)cudaFree(ctx->ws);
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  size_t want = bytes < (size_t)(4 << 20) ? (size_t)(4 << 20) : bytes;
+  st = cuda_status(cudaMalloc(&ctx->ws, want));
+  if (st != ROSAQ_OK) return st;
+  ctx->ws_bytes = want;
+  return ROSAQ_OK;
+}
+
+int run_gemm(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t, const int32_t *col_map,
+             __half *y, long long ldy, cudaStream_t s) {
+  if (ctx->impl == 1) return launch_linear_simt(ctx, x, M, ldx, t, col_map, y, ldy, s);
+  return launch_linear_tc(ctx, x, M, ldx, t, col_map, y, ldy, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *rosaq_strerror(int status) {
+  switch (status) {
+    case ROSAQ_OK: return "ok";
+    case ROSAQ_ERR_INVALID_ARG: return "invalid argument";
+    case ROSAQ_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case ROSAQ_ERR_ALIGNMENT: return "pointer or leading dimension not 16-byte aligned";
+    case ROSAQ_ERR_ALLOC: return "allocation failed";
+    case ROSAQ_ERR_CUDA: return "CUDA call failed";
+    case ROSAQ_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case ROSAQ_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    default: return "unknown status";
+  }
+}
+
+int rosaq_create(rosaq_ctx **out, int device) {
+  if (!out) return ROSAQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
+  if (device < 0 || device >= count) return ROSAQ_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  int st = cuda_status(cudaGetDeviceProperties(&prop, device));
+  if (st != ROSAQ_OK) return st;
+  if (prop.major != 10) return ROSAQ_ERR_UNSUPPORTED_ARCH;
+  DeviceGuard guard(device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  rosaq_ctx *ctx = new (std::nothrow) rosaq_ctx();
+  if (!ctx) return ROSAQ_ERR_ALLOC;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  ctx->wait_limit = 1ll << 26;
+  ctx->impl = 0;
+  st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), sizeof(int)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
+  if (st != ROSAQ_OK) {
+    if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    delete ctx;
+    return st;
+  }
+  *out = ctx;
+  return ROSAQ_OK;
+}
+
+int rosaq_destroy(rosaq_ctx *ctx) {
+  if (!ctx) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (guard.ok) {
+    (void)cudaDeviceSynchronize();
+    if (ctx->ws) (void)cudaFree(ctx->ws);
+    if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    (void)cudaGetLastError();
+  }
+  delete ctx;
+  return ROSAQ_OK;
+}
+
+int rosaq_last_status(rosaq_ctx *ctx, void *stream) {
+  if (!ctx) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int st = cuda_status(cudaStreamSynchronize(s));
+  if (st != ROSAQ_OK) return st;
+  int host = 0;
+  st = cuda_status(cudaMemcpy(&host, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != ROSAQ_OK) return st;
+  if (host != 0) {
+    st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
+    if (st != ROSAQ_OK) return st;
+  }
+  return host;
+}
+
+int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
+  if (!ctx) return 0;
+  int64_t prev = ctx->wait_limit;
+  if (iterations > 0) ctx->wait_limit = iterations;
+  return prev;
+}
+
+int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
+  if (!ctx) return 0;
+  int prev = ctx->impl;
+  if (impl == 0 || impl == 1) ctx->impl = impl;
+  return prev;
+}
+
+int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens, int d, int64_t ldx,
+                    int n_blocks, float *C, void *stream) {
+  if (!ctx || !X || !C) return ROSAQ_ERR_INVALID_ARG;
+  if (x_dtype != ROSAQ_F16 && x_dtype != ROSAQ_F32) return ROSAQ_ERR_INVALID_ARG;
+  if (n_tokens < 0 || d <= 0 || n_blocks <= 0 || ldx < d) return ROSAQ_ERR_INVALID_ARG;
+  if (d % n_blocks != 0 || d % 8 != 0 || (d / n_blocks) % 8 != 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(X) || !aligned16(C) || (ldx % 8) != 0) return ROSAQ_ERR_ALIGNMENT;
+  if (n_tokens == 0) return ROSAQ_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  return launch_cov(X, x_dtype, n_tokens, d, ldx, n_blocks, C, static_cast<cudaStream_t>(stream));
+}
+
+int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, int bits,
+                   int group, int k_salient, rosaq_weight **out, void *stream) {
+  if (!out) return ROSAQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !W) return ROSAQ_ERR_INVALID_ARG;
+  int st = check_quant_args(d_in, d_out, bits, group, k_salient);
+  if (st != ROSAQ_OK) return st;
+  if (!aligned16(W)) return ROSAQ_ERR_ALIGNMENT;
+  if (rot) {
+    if (!rot->q || rot->d != d_in || rot->n_blocks <= 0 || d_in % rot->n_blocks != 0) return ROSAQ_ERR_INVALID_ARG;
+    if (rot->q_dtype != ROSAQ_F32 && rot->q_dtype != ROSAQ_F16) return ROSAQ_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  rosaq_weight *w = new (std::nothrow) rosaq_weight();
+  if (!w) return ROSAQ_ERR_ALLOC;
+  w->group = group;
+  w->k_salient = k_salient;
+  w->device = ctx->device;
+  w->t = make_geometry(d_in, d_out, bits, k_salient / kGroup, (d_in - k_salient) / kGroup, 0);
+  float *Wp = nullptr;
+  st = alloc_blob(&w->t);
+  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Wp), sizeof(float) * (size_t)d_in * d_out));
+  if (st == ROSAQ_OK) {
+    if (rot)
+      st = launch_rotate_weights(rot->q, rot->q_dtype == ROSAQ_F32, d_in, rot->n_blocks, rot->perm,
+                                 static_cast<const __half *>(W), d_out, Wp, s);
+    else
+      st = launch_cast_weights(static_cast<const __half *>(W), d_in, d_out, Wp, s);
+  }
+  if (st == ROSAQ_OK) st = launch_quant_pack(Wp, w->t, s);
+  if (st == ROSAQ_OK) st = cuda_status(cudaStreamSynchronize(s));
+  if (Wp) (void)cudaFree(Wp);
+  if (st != ROSAQ_OK) {
+    if (w->t.blob) (void)cudaFree(w->t.blob);
+    delete w;
+    return st;
+  }
+  *out = w;
+  return ROSAQ_OK;
+}
+
+int rosaq_weight_export(rosaq_ctx *ctx, const rosaq_weight *w, uint32_t *qw, void *scales_f16, void *zeros_f16,
+                        void *salient_f16, void *stream) {
+  if (!ctx || !w) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  return launch_export(w->t, qw, static_cast<__half *>(scales_f16), static_cast<__half *>(zeros_f16),
+                       static_cast<__half *>(salient_f16), static_cast<cudaStream_t>(stream));
+}
+
+int rosaq_weight_import(rosaq_ctx *ctx, int d_in, int d_out, int bits, int group, int k_salient,
+                        const uint32_t *qw, const void *scales_f16, const void *zeros_f16, const void *salient_f16,
+                        rosaq_weight **out, void *stream) {
+  if (!out) return ROSAQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx) return ROSAQ_ERR_INVALID_ARG;
+  int st = check_quant_args(d_in, d_out, bits, group, k_salient);
+  if (st != ROSAQ_OK) return st;
+  if (k_salient > 0 && !salient_f16) return ROSAQ_ERR_INVALID_ARG;
+  if (k_salient < d_in && (!qw || !scales_f16 || !zeros_f16)) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rosaq_weight *w = new (std::nothrow) rosaq_weight();
+  if (!w) return ROSAQ_ERR_ALLOC;
+  w->group = group;
+  w->k_salient = k_salient;
+  w->device = ctx->device;
+  w->t = make_geometry(d_in, d_out, bits, k_salient / kGroup, (d_in - k_salient) / kGroup, 0);
+  st = alloc_blob(&w->t);
+  if (st == ROSAQ_OK)
+    st = launch_import(w->t, qw, static_cast<const __half *>(scales_f16), static_cast<const __half *>(zeros_f16),
+                       static_cast<const __half *>(salient_f16), s);
+  if (st == ROSAQ_OK) st = cuda_status(cudaStreamSynchronize(s));
+  if (st != ROSAQ_OK) {
+    if (w->t.blob) (void)cudaFree(w->t.blob);
+    delete w;
+    return st;
+  }
+  *out = w;
+  return ROSAQ_OK;
+}
+
+int rosaq_weight_free(rosaq_weight *w) {
+  if (!w) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(w->device);
+  if (guard.ok && w->t.blob) {
+    (void)cudaFree(w->t.blob);
+    (void)cudaGetLastError();
+  }
+  delete w;
+  return ROSAQ_OK;
+}
+
+int rosaq_weight_info(const rosaq_weight *w, int *d_in, int *d_out, int *bits, int *group, int *k_salient,
+                      int64_t *device_bytes) {
+  if (!w) return ROSAQ_ERR_INVALID_ARG;
+  if (d_in) *d_in = w->t.d_in;
+  if (d_out) *d_out = w->t.d_out;
+  if (bits) *bits = w->t.bits;
+  if (group) *group = w->group;
+  if (k_salient) *k_salient = w->k_salient;
+  if (device_bytes) *device_bytes = w->t.bytes;
+  return ROSAQ_OK;
+}
+
+int rosaq_rotation_create(rosaq_ctx *ctx, const rosaq_rot *rot, rosaq_rotation **out, void *stream) {
+  if (!out) return ROSAQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !rot || !rot->q) return ROSAQ_ERR_INVALID_ARG;
+  if (rot->q_dtype != ROSAQ_F16) return ROSAQ_ERR_INVALID_ARG;
+  if (rot->d <= 0 || rot->n_blocks <= 0 || rot->d % rot->n_blocks != 0) return ROSAQ_ERR_INVALID_ARG;
+  const int dh = rot->d / rot->n_blocks;
+  if (dh % kGroup != 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(rot->q)) return ROSAQ_ERR_ALIGNMENT;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rosaq_rotation *r = new (std::nothrow) rosaq_rotation();
+  if (!r) return ROSAQ_ERR_ALLOC;
+  r->d = rot->d;
+  r->device = ctx->device;
+  r->col_map = nullptr;
+  const int bg = dh / kGroup;
+  r->t = make_geometry(rot->d, rot->d, 4, bg, 0, rot->n_blocks == 1 ? 0 : bg);
+  int st = alloc_blob(&r->t);
+  if (st == ROSAQ_OK) st = launch_rotation_tiles(static_cast<const __half *>(rot->q), rot->d, rot->n_blocks, r->t, s);
+  if (st == ROSAQ_OK && rot->perm) {
+    st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&r->col_map), sizeof(int32_t) * rot->d));
+    if (st == ROSAQ_OK) st = launch_invert_perm(rot->perm, rot->d, r->col_map, s);
+  }
+  if (st == ROSAQ_OK) st = cuda_status(cudaStreamSynchronize(s));
+  if (st != ROSAQ_OK) {
+    if (r->t.blob) (void)cudaFree(r->t.blob);
+    if (r->col_map) (void)cudaFree(r->col_map);
+    delete r;
+    return st;
+  }
+  *out = r;
+  return ROSAQ_OK;
+}
+
+int rosaq_rotation_free(rosaq_rotation *r) {
+  if (!r) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(r->device);
+  if (guard.ok) {
+    if (r->t.blob) (void)cudaFree(r->t.blob);
+    if (r->col_map) (void)cudaFree(r->col_map);
+    (void)cudaGetLastError();
+  }
+  delete r;
+  return ROSAQ_OK;
+}
+
+static int check_act(const void *p, int M, int64_t ld, int d) {
+  if (!p || M <= 0 || ld < d) return ROSAQ_ERR_INVALID_ARG;
+  if (!aligned16(p) || (ld % 8) != 0) return ROSAQ_ERR_ALIGNMENT;
+  return ROSAQ_OK;
+}
+
+int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r, void *x_rot,
+                 int64_t ldxr, void *stream) {
+  if (!ctx || !r) return ROSAQ_ERR_INVALID_ARG;
+  int st = check_act(x, M, ldx, r->d);
+  if (st == ROSAQ_OK) st = check_act(x_rot, M, ldxr, r->d);
+  if (st != ROSAQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  return run_gemm(ctx, static_cast<const __half *>(x), M, ldx, r->t, r->col_map, static_cast<__half *>(x_rot), ldxr,
+                  static_cast<cudaStream_t>(stream));
+}
+
+int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r, const rosaq_weight *w,
+                 void *y, int64_t ldy, void *stream) {
+  if (!ctx || !w) return ROSAQ_ERR_INVALID_ARG;
+  int st = check_act(x, M, ldx, w->t.d_in);
+  if (st == ROSAQ_OK) st = check_act(y, M, ldy, w->t.d_out);
+  if (st != ROSAQ_OK) return st;
+  if (r && r->d != w->t.d_in) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __half *xin = static_cast<const __half *>(x);
+  long long ld = ldx;
+  if (r) {
+    st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
+    if (st != ROSAQ_OK) return st;
+    st = run_gemm(ctx, xin, M, ldx, r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d, s);
+    if (st != ROSAQ_OK) return st;
+    xin = static_cast<const __half *>(ctx->ws);
+    ld = r->d;
+  }
+  return run_gemm(ctx, xin, M, ld, w->t, nullptr, static_cast<__half *>(y), ldy, s);
+}
+
+}  // extern "C"

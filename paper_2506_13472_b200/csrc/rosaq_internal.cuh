@@ -1,0 +1,224 @@
+// Internal declarations shared by the translation units of librosaq (CUDA side only).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rosaq.h"
+
+namespace rosaq {
+
+// ------------------------------------------------------------------------------------
+// Tiled operand layout.
+//
+// A [d_in][d_out] matrix that the GEMM kernels stream is cut into tiles of 128 input
+// channels (one quantization group, Section 3: "a group consists of 128 channels") by
+// 128 output columns.  All tiles of one column tile are contiguous, in input-channel
+// order, so that a CTA walking down K reads one linear stretch of memory; every tile is
+// a self-contained blob that one bulk copy brings into shared memory:
+//
+//   fp16 tile   (salient group of Eq. 3, or a tile of a rotation matrix)      32768 B
+//     element (k, n) at byte ((k/8)*128 + n)*16 + (k%8)*2
+//   INT4 tile                                                         8192 + 512 B
+//     16-byte chunk j = k/32 of column n at (j*128 + n)*16; inside it word w = (k%32)/8;
+//     inside the word the code of k%8 = i sits in nibble (i even ? i/2 : 4 + i/2), so that
+//     (word & 0x000f000f) is the pair (k, k+1) laid out as two fp16 mantissas
+//   INT3 tile                                                         6144 + 512 B
+//     12 words per column: word index wl = (k/32)*3 + ((k%32)/10) for k%32 < 30, the code of
+//     i = k%32 at bit 3*((i%10)/2) + 16*(i%2); codes 30 and 31 of each 32 are spread over bit
+//     15 (code 30) and bit 31 (code 31) of the three words, one bit per word;
+//     word wl of column n at ((wl/4)*128 + n)*16 + (wl%4)*4
+//   quantized tiles end with 128 x {fp16 scale, fp16 zero} (column n at codes_bytes + 4n)
+//
+// Column k of TMEM then holds the fp16 pair (2k, 2k+1), which is what the chunk order
+// above delivers after the in-register dequantisation.
+// ------------------------------------------------------------------------------------
+constexpr int kTileN = 128;
+constexpr int kGroup = 128;
+constexpr int kFp16TileBytes = kGroup * kTileN * 2;
+constexpr int kInt4CodeBytes = kGroup * kTileN / 2;
+constexpr int kInt3CodeBytes = kGroup * kTileN * 3 / 8;
+constexpr int kScaleBytes = kTileN * 4;
+
+__host__ __device__ inline int quant_tile_bytes(int bits) {
+  return (bits == 4 ? kInt4CodeBytes : kInt3CodeBytes) + kScaleBytes;
+}
+__host__ __device__ inline int quant_code_bytes(int bits) {
+  return bits == 4 ? kInt4CodeBytes : kInt3CodeBytes;
+}
+
+struct TiledOperand {
+  uint8_t *blob;        // device
+  int d_in, d_out;      // logical sizes
+  int n_tiles;          // ceil(d_out / 128); the last tile is zero padded
+  int bits;             // 3 or 4 (ignored when g_quant == 0)
+  int g_fp16;           // leading fp16 groups per column tile
+  int g_quant;          // quantized groups that follow
+  int block_groups;     // 0: every column tile spans all of d_in.  >0: block-diagonal operand whose
+                        // column tile t only holds the `block_groups` groups of its own diagonal
+                        // block (then g_fp16 == block_groups, g_quant == 0)
+  long long tile_stride;  // bytes between consecutive column tiles
+  long long bytes;        // total
+};
+
+__host__ __device__ inline int groups_per_tile(const TiledOperand &t) { return t.g_fp16 + t.g_quant; }
+
+// byte offset of local group lg of column tile nt
+__host__ __device__ inline long long tile_offset(const TiledOperand &t, int nt, int lg) {
+  long long o = (long long)nt * t.tile_stride;
+  if (lg < t.g_fp16) return o + (long long)lg * kFp16TileBytes;
+  return o + (long long)t.g_fp16 * kFp16TileBytes + (long long)(lg - t.g_fp16) * quant_tile_bytes(t.bits);
+}
+
+// first input channel that local group lg of column tile nt multiplies
+__host__ __device__ inline int group_k0(const TiledOperand &t, int nt, int lg) {
+  if (t.block_groups == 0) return lg * kGroup;
+  int tiles_per_block = t.block_groups;  // square blocks: block size = block_groups * 128 columns
+  return ((nt / tiles_per_block) * t.block_groups + lg) * kGroup;
+}
+
+// ---- positions inside a tile -----------------------------------------------------------
+__host__ __device__ inline int fp16_tile_byte(int k, int n) { return ((k >> 3) * kTileN + n) * 16 + (k & 7) * 2; }
+
+__host__ __device__ inline void int4_pos(int k, int n, int *byte, int *shift) {
+  int j = k >> 5, w = (k & 31) >> 3, i = k & 7;
+  int nib = (i & 1) ? 4 + (i >> 1) : (i >> 1);
+  *byte = (j * kTileN + n) * 16 + w * 4;
+  *shift = nib * 4;
+}
+
+// INT3: codes 0..29 of each 32 occupy one 3-bit field; codes 30/31 are bit-sliced (see above).
+__host__ __device__ inline int int3_word_byte(int wl, int n) { return ((wl >> 2) * kTileN + n) * 16 + (wl & 3) * 4; }
+__host__ __device__ inline void int3_field(int i /*0..29*/, int *word, int *shift) {
+  *word = i / 10;
+  *shift = 3 * ((i % 10) >> 1) + 16 * (i & 1);
+}
+
+#ifdef __CUDACC__
+// ---- per-column access to a quantized tile (code words of one output column in registers) ----
+template <int kBits>
+__device__ __forceinline__ void put_code(uint32_t *words, int k, uint32_t code) {
+  if (kBits == 4) {
+    int i = k & 7;
+    int nib = (i & 1) ? 4 + (i >> 1) : (i >> 1);
+    words[k >> 3] |= code << (nib * 4);
+  } else {
+    int set = k >> 5, i = k & 31;
+    if (i < 30) {
+      words[set * 3 + i / 10] |= code << (3 * ((i % 10) >> 1) + 16 * (i & 1));
+    } else {
+      int bit = 15 + 16 * (i - 30);
+#pragma unroll
+      for (int b = 0; b < 3; ++b) words[set * 3 + b] |= ((code >> b) & 1u) << bit;
+    }
+  }
+}
+
+template <int kBits>
+__device__ __forceinline__ uint32_t get_code(const uint32_t *words, int k) {
+  if (kBits == 4) {
+    int i = k & 7;
+    int nib = (i & 1) ? 4 + (i >> 1) : (i >> 1);
+    return (words[k >> 3] >> (nib * 4)) & 0xf;
+  } else {
+    int set = k >> 5, i = k & 31;
+    if (i < 30) return (words[set * 3 + i / 10] >> (3 * ((i % 10) >> 1) + 16 * (i & 1))) & 0x7;
+    int bit = 15 + 16 * (i - 30);
+    uint32_t c = 0;
+#pragma unroll
+    for (int b = 0; b < 3; ++b) c |= ((words[set * 3 + b] >> bit) & 1u) << b;
+    return c;
+  }
+}
+
+template <int kBits>
+__device__ __forceinline__ void store_quant_tile_column(uint8_t *tile, int n, const uint32_t *words, __half scale,
+                                                        __half zero) {
+  constexpr int kWords = kBits == 4 ? 16 : 12;
+#pragma unroll
+  for (int j = 0; j < kWords / 4; ++j)
+    *reinterpret_cast<uint4 *>(tile + (j * kTileN + n) * 16) =
+        make_uint4(words[4 * j], words[4 * j + 1], words[4 * j + 2], words[4 * j + 3]);
+  *reinterpret_cast<uint32_t *>(tile + quant_code_bytes(kBits) + n * 4) =
+      (uint32_t)__half_as_ushort(scale) | ((uint32_t)__half_as_ushort(zero) << 16);
+}
+
+template <int kBits>
+__device__ __forceinline__ void load_quant_tile_column(const uint8_t *tile, int n, uint32_t *words, __half *scale,
+                                                       __half *zero) {
+  constexpr int kWords = kBits == 4 ? 16 : 12;
+#pragma unroll
+  for (int j = 0; j < kWords / 4; ++j) {
+    uint4 v = *reinterpret_cast<const uint4 *>(tile + (j * kTileN + n) * 16);
+    words[4 * j] = v.x, words[4 * j + 1] = v.y, words[4 * j + 2] = v.z, words[4 * j + 3] = v.w;
+  }
+  uint32_t sz = *reinterpret_cast<const uint32_t *>(tile + quant_code_bytes(kBits) + n * 4);
+  *scale = __ushort_as_half((unsigned short)(sz & 0xffff));
+  *zero = __ushort_as_half((unsigned short)(sz >> 16));
+}
+
+#endif  // __CUDACC__
+
+// ---- handles -----------------------------------------------------------------------------
+}  // namespace rosaq
+
+struct rosaq_ctx {
+  int device;
+  int sm_count;
+  int *d_status;       // device status word (0 or ROSAQ_ERR_TIMEOUT)
+  void *ws;            // rotated-activation workspace
+  size_t ws_bytes;
+  long long wait_limit;
+  int impl;            // 0 tensor-core, 1 CUDA-core
+};
+
+struct rosaq_weight {
+  rosaq::TiledOperand t;
+  int group, k_salient, device;
+};
+
+struct rosaq_rotation {
+  rosaq::TiledOperand t;
+  int32_t *col_map;    // device [d] or nullptr: rotated column p is stored at position col_map[p]
+  int d, device;
+};
+
+namespace rosaq {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
+    if (ok && prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    if (!ok) (void)cudaGetLastError();
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) (void)cudaSetDevice(prev);
+  }
+};
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// launchers implemented in the other translation units; all return a rosaq_status
+int launch_rotate_weights(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
+                          const __half *W, int d_out, float *Wp, cudaStream_t s);
+int launch_cast_weights(const __half *W, int d_in, int d_out, float *Wp, cudaStream_t s);
+int launch_quant_pack(const float *Wp, const TiledOperand &t, cudaStream_t s);
+int launch_export(const TiledOperand &t, uint32_t *qw, __half *scales, __half *zeros, __half *salient,
+                  cudaStream_t s);
+int launch_import(const TiledOperand &t, const uint32_t *qw, const __half *scales, const __half *zeros,
+                  const __half *salient, cudaStream_t s);
+int launch_rotation_tiles(const __half *q, int d, int n_blocks, const TiledOperand &t, cudaStream_t s);
+int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, cudaStream_t s);
+int launch_cov_fma(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
+                   cudaStream_t s);
+int launch_cov(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
+               cudaStream_t s);
+int launch_linear_simt(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
+                       const int32_t *col_map, __half *y, long long ldy, cudaStream_t s);
+int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
+                     const int32_t *col_map, __half *y, long long ldy, cudaStream_t s);
+
+}  // namespace rosaq

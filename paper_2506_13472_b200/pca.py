@@ -1,0 +1,33 @@
+"""Host-side step between rosaq_calib_cov and rosaq_quantize: C = R Lambda R^T (Eq. 4).
+
+The eigensolve is deliberately outside the C ABI (R is an input of the device calls);
+this helper is what the benchmark and a user of the library call to get R from the
+Gram matrix that rosaq_calib_cov produced.  LAPACK (through numpy) in fp64.
+"""
+import numpy as np
+
+
+def eigh_descending(Cm):
+    """(lambda, R): eigenvalues in descending order (Section 3.2: the largest are the salient
+    ones), R[:, j] the unit eigenvector of lambda[j], sign chosen so that its largest-magnitude
+    entry is positive (eigenvectors are only defined up to sign)."""
+    Cm = np.asarray(Cm, dtype=np.float64)
+    Cm = 0.5 * (Cm + Cm.T)
+    lam, V = np.linalg.eigh(Cm)
+    order = np.argsort(-lam, kind="stable")
+    lam, V = lam[order], V[:, order]
+    big = np.argmax(np.abs(V), axis=0)
+    sgn = np.sign(V[big, np.arange(V.shape[1])])
+    sgn[sgn == 0] = 1.0
+    return lam, V * sgn[None, :]
+
+
+def headwise_rotation(C_blocks):
+    """Head-wise PCA (Section 3.1.1, Eq. 6): one eigendecomposition per head block plus the
+    global column order by descending eigenvalue, so that the first K columns of
+    R = blockdiag(R_1..R_H)[:, perm] are the K most principal directions over all heads.
+    Returns (Rb [H][dh][dh] fp64, perm [H*dh] int32, lambdas [H][dh])."""
+    lams, Rs = zip(*[eigh_descending(Cb) for Cb in np.asarray(C_blocks)])
+    lams = np.asarray(lams)
+    perm = np.argsort(-lams.reshape(-1), kind="stable").astype(np.int32)
+    return np.ascontiguousarray(Rs), perm, lams

@@ -1,0 +1,70 @@
+"""Shared builders for the parity tests: seeded configs, oracle-side expectations, comparisons."""
+import functools
+
+import numpy as np
+
+from oracle import rosaq_oracle as orc
+from paper_2506_13472_b200 import synth
+
+REL_TOL_Y = 2e-3   # ||y - y_ref||_F / ||y_ref||_F, the bound the path is specified to
+
+
+def rel_fro(a, b):
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+@functools.lru_cache(maxsize=None)
+def config_tiny(seed=0):
+    """Config 1: d_in = d_out = 512, 256 calibration tokens (fp32), spectrum i^-1.2, QR mix,
+    4 outlier input rows x20, M = 4.  R = oracle Jacobi eigenvectors of X^T X."""
+    d = 512
+    law = synth.ActivationLaw(d, 1.2, seed, "tiny", mix="qr")
+    X = law.sample(256, "calib", np.float32)
+    lam, V = orc.eigh_jacobi(orc.cov(X))
+    W = synth.weights(d, d, seed, "tiny", sigma=0.02, outlier_rows=4, outlier_scale=20.0)
+    x = law.sample(4, "x", np.float16)
+    return dict(X=X, lam=lam, R64=V, R32=V.astype(np.float32), R16=V.astype(np.float16), W=W, x=x, d=d)
+
+
+@functools.lru_cache(maxsize=None)
+def config_headwise(seed=3, heads=4, head_dim=128, n_tokens=512, d_out=384, M=5):
+    """Small head-wise case (Eq. 6): per-head PCA blocks + the global descending permutation."""
+    law = synth.HeadwiseActivationLaw(heads, head_dim, seed, "hw")
+    X = law.sample(n_tokens, "calib", np.float16)
+    Cb = orc.cov(X, n_blocks=heads)
+    lams, Vs = zip(*[orc.eigh_jacobi(Cb[h]) for h in range(heads)])
+    Rb, perm = orc.assemble_headwise_rotation(np.array(lams), np.array(Vs))
+    W = synth.weights(heads * head_dim, d_out, seed, "hw", outlier_frac=0.01)
+    x = law.sample(M, "x", np.float16)
+    return dict(X=X, Rb64=Rb, Rb32=Rb.astype(np.float32), Rb16=Rb.astype(np.float16), perm=perm, W=W, x=x,
+                heads=heads, head_dim=head_dim)
+
+
+def oracle_quantized(W16, R32_blocks, perm, bits, k_salient, cols=None, group=128):
+    """Oracle expectation for rosaq_quantize on the listed columns: dict with packed qw too."""
+    d_in, d_out = W16.shape
+    cols = np.arange(d_out, dtype=np.int32) if cols is None else np.asarray(cols, np.int32)
+    if R32_blocks is None:
+        Wp = W16[:, cols].astype(np.float32)
+    else:
+        Wp = orc.rotate_weights_f32(R32_blocks, W16, perm, cols)
+    qd = orc.quantize(Wp, bits, group, k_salient)
+    qd["qw"] = orc.pack(qd["codes"], bits) if qd["codes"].shape[0] else np.zeros((0, cols.size), np.uint32)
+    qd["cols"] = cols
+    return qd
+
+
+def assert_export_matches(exported, qd):
+    """Bit-exact comparison of a GPU export (numpy arrays) with the oracle dict on qd['cols']."""
+    cols = qd["cols"]
+    got_qw = exported["qw"].view(np.uint32)[:, cols]
+    assert np.array_equal(exported["salient"].view(np.uint16)[:, cols], qd["salient"].view(np.uint16)), "salient"
+    assert np.array_equal(exported["scales"].view(np.uint16)[:, cols], qd["scales"].view(np.uint16)), "scales"
+    assert np.array_equal(exported["zeros"].view(np.uint16)[:, cols], qd["zeros"].view(np.uint16)), "zeros"
+    assert np.array_equal(got_qw, qd["qw"]), "packed codes"
+
+
+def export_to_numpy(exported):
+    return {k: v.cpu().numpy() for k, v in exported.items()}

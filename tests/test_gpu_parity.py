@@ -1,0 +1,215 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Integer / byte results (packed codes, scales, zeros, salient fp16 bits) must be bit-exact.
+y must satisfy ||y - y_ref||_F / ||y_ref||_F <= 2e-3 against the oracle's fp64 forward on the
+same dequantised weights.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rosaq_oracle as orc
+from paper_2506_13472_b200 import binding as rb
+from paper_2506_13472_b200 import pca, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = rb.Context(0)
+    yield c
+    c.close()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def check_status(ctx):
+    assert ctx.last_status() == rb.ROSAQ_OK
+
+
+# --------------------------------------------------------------------------- quantize
+@pytest.mark.parametrize("bits", [4, 3])
+def test_quantize_tiny_config_bit_exact(ctx, bits):
+    c = H.config_tiny()
+    w = ctx.quantize(dev(c["W"]), dev(c["R32"]), bits=bits, k_salient=128)
+    H.assert_export_matches(H.export_to_numpy(w.export()), H.oracle_quantized(c["W"], c["R32"], None, bits, 128))
+    check_status(ctx)
+
+
+@pytest.mark.parametrize("bits,k_salient,d_out", [(4, 0, 200), (3, 0, 129), (4, 256, 8), (3, 256, 128), (4, 128, 1)])
+def test_quantize_no_rotation_ragged_and_degenerate(ctx, bits, k_salient, d_out):
+    W = synth.weights(256, d_out, seed=21, key=f"nr{d_out}", outlier_rows=3, outlier_scale=20.0)
+    W[130:140, 0] = 0.25          # constant stretch; column 0 of group 1 below gets fully constant
+    W[128:256, d_out - 1] = 0.125 # a constant group: range floor, zero-point clamp
+    w = ctx.quantize(dev(W), None, bits=bits, k_salient=k_salient)
+    assert (w.d_in, w.d_out, w.bits, w.k_salient) == (256, d_out, bits, k_salient)
+    H.assert_export_matches(H.export_to_numpy(w.export()), H.oracle_quantized(W, None, None, bits, k_salient))
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+def test_quantize_headwise_blockdiag_with_permutation(ctx, bits):
+    c = H.config_headwise()
+    w = ctx.quantize(dev(c["W"]), dev(c["Rb32"]), dev(c["perm"]), bits=bits, k_salient=128)
+    H.assert_export_matches(H.export_to_numpy(w.export()),
+                            H.oracle_quantized(c["W"], c["Rb32"], c["perm"], bits, 128))
+    # Eq. 6 == Eq. 7: the same weight through the dense path fed blockdiag . P
+    Rd = orc.dense_from_blocks(c["Rb32"], c["perm"])
+    w2 = ctx.quantize(dev(c["W"]), dev(Rd), bits=bits, k_salient=128)
+    a, b = H.export_to_numpy(w.export()), H.export_to_numpy(w2.export())
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+def test_import_export_round_trip(ctx, bits):
+    rng = np.random.default_rng(5)
+    d_in, d_out, K = 512, 300, 128
+    nq = d_in - K
+    codes = rng.integers(0, 2 ** bits, (nq, d_out)).astype(np.uint8)
+    qw = orc.pack(codes, bits)
+    sc = rng.uniform(1e-3, 1e-1, (nq // 128, d_out)).astype(np.float16)
+    zr = rng.integers(0, 2 ** bits, (nq // 128, d_out)).astype(np.float16)
+    sal = rng.standard_normal((K, d_out)).astype(np.float16)
+    w = ctx.weight_import(d_in, d_out, bits, 128, K, dev(qw.view(np.int32)), dev(sc), dev(zr), dev(sal))
+    e = H.export_to_numpy(w.export())
+    assert np.array_equal(e["qw"].view(np.uint32), qw)
+    assert np.array_equal(e["scales"], sc) and np.array_equal(e["zeros"], zr) and np.array_equal(e["salient"], sal)
+
+
+# --------------------------------------------------------------------------- linear
+def run_linear_case(ctx, x16, W16, Rb32, Rb16, perm, bits, k_salient, impl):
+    """quantize on the GPU, check codes, then y against the oracle forward on the same inputs."""
+    ctx.set_linear_impl(impl)
+    try:
+        w = ctx.quantize(dev(W16), None if Rb32 is None else dev(Rb32), None if perm is None else dev(perm),
+                         bits=bits, k_salient=k_salient)
+        qd = H.oracle_quantized(W16, Rb32, perm, bits, k_salient)
+        H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+        rot = None if Rb16 is None else ctx.rotation_create(dev(Rb16), None if perm is None else dev(perm))
+        y = ctx.linear(dev(x16), w, rot).cpu().numpy()
+        y_ref, xr_ref = orc.forward(x16, qd, Rb16, perm, return_xrot=True)
+        assert np.all(np.isfinite(y))
+        assert H.rel_fro(y, y_ref) <= H.REL_TOL_Y
+        if rot is not None:
+            xr = ctx.rotate(dev(x16), rot).cpu().numpy()
+            assert H.rel_fro(xr, xr_ref) <= 1e-3
+            # pre-rotated input through the GEMM stage alone gives the same y bits
+            y2 = ctx.linear(dev(xr), w, None).cpu().numpy()
+            assert np.array_equal(y2.view(np.uint16), y.view(np.uint16))
+        check_status(ctx)
+    finally:
+        ctx.set_linear_impl(0)
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("bits", [4, 3])
+def test_linear_tiny_config(ctx, bits, impl):
+    c = H.config_tiny()
+    run_linear_case(ctx, c["x"], c["W"], c["R32"], c["R16"], None, bits, 128, impl)
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("bits", [4, 3])
+def test_linear_headwise(ctx, bits, impl):
+    c = H.config_headwise()
+    run_linear_case(ctx, c["x"], c["W"], c["Rb32"], c["Rb16"], c["perm"], bits, 128, impl)
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("M,d_in,d_out,bits,k_salient", [
+    (1, 256, 8, 4, 128), (3, 256, 136, 3, 0), (17, 384, 128, 4, 384), (64, 1024, 640, 4, 128),
+    (130, 512, 256, 3, 128), (257, 256, 200, 4, 0)])
+def test_linear_shapes_no_rotation(ctx, M, d_in, d_out, bits, k_salient, impl):
+    W = synth.weights(d_in, d_out, seed=31, key=f"s{d_in}x{d_out}", outlier_frac=0.01)
+    x = synth.rng_for(31, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+    run_linear_case(ctx, x, W, None, None, None, bits, k_salient, impl)
+
+
+def test_linear_strided_activations_and_output(ctx):
+    c = H.config_tiny()
+    w = ctx.quantize(dev(c["W"]), dev(c["R32"]), bits=4, k_salient=128)
+    qd = H.oracle_quantized(c["W"], c["R32"], None, 4, 128)
+    xbuf = torch.zeros((4, 512 + 64), dtype=torch.float16, device="cuda")
+    xbuf[:, :512] = dev(c["x"])
+    ybuf = torch.full((4, 512 + 8), 7.0, dtype=torch.float16, device="cuda")
+    rot = ctx.rotation_create(dev(c["R16"]))
+    ctx.linear(xbuf[:, :512], w, rot, out=ybuf[:, :512])
+    assert H.rel_fro(ybuf[:, :512].cpu().numpy(), orc.forward(c["x"], qd, c["R16"])) <= H.REL_TOL_Y
+    assert torch.all(ybuf[:, 512:] == 7.0)       # nothing written past d_out
+
+
+def test_special_case_all_salient_is_plain_fp16_gemm(ctx):
+    rng = np.random.default_rng(12)
+    W = (rng.standard_normal((256, 128)) * 0.02).astype(np.float16)
+    x = rng.standard_normal((9, 256)).astype(np.float16)
+    w = ctx.quantize(dev(W), None, bits=4, k_salient=256)
+    y = ctx.linear(dev(x), w).cpu().numpy()
+    ref = x.astype(np.float64) @ W.astype(np.float64)
+    assert H.rel_fro(y, ref) <= 1e-3
+
+
+# --------------------------------------------------------------------------- calib_cov
+def cov_tolerance(Cref, n_tokens):
+    """fp32 accumulation of exact (fp16 x fp16) or once-rounded (fp32) products: the error of a
+    length-N fp32 sum is bounded by ~N u sum|terms| and is ~sqrt(N) u in practice; by
+    Cauchy-Schwarz sum_t |x_ti x_tj| <= sqrt(C_ii C_jj)."""
+    dg = np.sqrt(np.clip(np.diagonal(Cref, axis1=-2, axis2=-1), 0, None))
+    return 2.0 ** -24 * (4.0 * np.sqrt(n_tokens) + 8.0) * dg[..., :, None] * dg[..., None, :]
+
+
+@pytest.mark.parametrize("dtype,n_tokens,d,n_blocks", [
+    (np.float32, 256, 512, 1), (np.float16, 300, 264, 1), (np.float16, 1000, 512, 4), (np.float16, 64, 8, 1)])
+def test_calib_cov_matches_oracle_and_accumulates(ctx, dtype, n_tokens, d, n_blocks):
+    law = synth.ActivationLaw(d, 1.0, seed=41, key=f"cov{d}", mix="householder")
+    X = law.sample(n_tokens, "X", dtype)
+    dh = d // n_blocks
+    Cg = torch.zeros((n_blocks, dh, dh), dtype=torch.float32, device="cuda")
+    half = n_tokens // 2 // 8 * 8
+    Xd = dev(X)
+    ctx.calib_cov(Xd[:half], Cg, n_blocks)        # two chunks: C accumulates
+    ctx.calib_cov(Xd[half:], Cg, n_blocks)
+    check_status(ctx)
+    Cref = orc.cov(X, n_blocks).reshape(n_blocks, dh, dh)
+    got = Cg.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - Cref) <= cov_tolerance(Cref, n_tokens) + 1e-30)
+    assert np.array_equal(got, np.swapaxes(got, -1, -2))          # both triangles written, symmetric
+
+
+def test_pca_helper_gives_valid_eigenpairs_from_gpu_cov(ctx):
+    c = H.config_tiny()
+    Cg = torch.zeros((512, 512), dtype=torch.float32, device="cuda")
+    ctx.calib_cov(dev(c["X"]), Cg)
+    lam, R = pca.eigh_descending(Cg.cpu().numpy())
+    C64 = orc.cov(c["X"])
+    nC = np.linalg.norm(C64)
+    assert np.all(np.diff(lam) <= 1e-9 * nC)
+    assert np.abs(R.T @ R - np.eye(512)).max() <= 1e-10
+    assert np.abs(C64 @ R - R * lam[None, :]).max() <= 1e-5 * nC
+    assert np.allclose(lam[:64], c["lam"][:64], rtol=1e-4)
+
+
+# --------------------------------------------------------------------------- argument errors
+def test_argument_errors_are_codes_not_faults(ctx):
+    W = torch.zeros((256, 128), dtype=torch.float16, device="cuda")
+    with pytest.raises(rb.RosaqError) as e:
+        ctx.quantize(W, None, bits=5)
+    assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+    with pytest.raises(rb.RosaqError) as e:
+        ctx.quantize(W, None, bits=4, k_salient=64)
+    assert e.value.status == rb.ROSAQ_ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(rb.RosaqError) as e:
+        ctx.quantize(torch.zeros((200, 128), dtype=torch.float16, device="cuda"), None)
+    assert e.value.status == rb.ROSAQ_ERR_UNSUPPORTED_SHAPE
+    w = ctx.quantize(W, None, bits=4, k_salient=128)
+    x = torch.zeros((4, 264), dtype=torch.float16, device="cuda")
+    with pytest.raises(rb.RosaqError) as e:
+        ctx.linear(x[:, 1:257], w)                          # misaligned pointer
+    assert e.value.status == rb.ROSAQ_ERR_ALIGNMENT
+    with pytest.raises(rb.RosaqError) as e:
+        ctx.linear(torch.zeros((4, 128), dtype=torch.float16, device="cuda"), w)   # ldx < d_in
+    assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+    assert ctx.last_status() == rb.ROSAQ_OK
