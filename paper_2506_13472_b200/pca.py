@@ -19,7 +19,7 @@ def eigh_descending(Cm):
     big = np.argmax(np.abs(V), axis=0)
     sgn = np.sign(V[big, np.arange(V.shape[1])])
     sgn[sgn == 0] = 1.0
-    return lam, V * sgn[None, :]
+    return lam, np.ascontiguousarray(V * sgn[None, :])
 
 
 def headwise_rotation(C_blocks):
