@@ -31,3 +31,18 @@ def headwise_rotation(C_blocks):
     lams = np.asarray(lams)
     perm = np.argsort(-lams.reshape(-1), kind="stable").astype(np.int32)
     return np.ascontiguousarray(Rs), perm, lams
+
+
+def eigh_descending_device(C_dev):
+    """Same contract as eigh_descending, computed in fp64 on the device the Gram matrix lives on
+    (a library eigensolver; used when d is in the thousands).  Returns a torch fp64 tensor R."""
+    import torch
+    Cm = C_dev.to(torch.float64)
+    Cm = 0.5 * (Cm + Cm.T)
+    lam, V = torch.linalg.eigh(Cm)
+    order = torch.argsort(lam, descending=True, stable=True)
+    V = V[:, order]
+    big = torch.argmax(V.abs(), dim=0)
+    sgn = torch.sign(V[big, torch.arange(V.shape[1], device=V.device)])
+    sgn[sgn == 0] = 1.0
+    return (V * sgn[None, :]).contiguous()
