@@ -84,7 +84,7 @@ const char *rosaq_strerror(int status);
 int rosaq_last_status(rosaq_ctx *ctx, void *stream);
 
 /* Test hook: upper bound, in polling iterations, of every device-side wait
- * (default 1<<26; a positive value replaces it).  Returns the previous value. */
+ * (default 1<<20; a positive value replaces it).  Returns the previous value. */
 int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
 
 /* Selects the rosaq_linear / rosaq_rotate implementation: 0 = tensor-core path

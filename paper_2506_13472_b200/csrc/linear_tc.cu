@@ -1,11 +1,630 @@
-// Tensor-core implementation of the GEMM stage (placeholder dispatch while the tcgen05 kernel is brought up).
+// Tensor-core implementation of the GEMM stage  y = x' . W^  (Eq. 3; Eq. 6 for a block-diagonal
+// rotation operand) for sm_100a: tcgen05.mma with the weight operand dequantised in registers
+// and fed from tensor memory.
+//
+// Mapping.  The MMA computes D[n][m] = sum_k A[n][k] * B[m][k] with
+//   A = one 128-column tile of the weights (MMA-M = 128 output columns), written to TMEM by the
+//       dequantisation warps (lane = output column, one 32-bit TMEM column = the fp16 pair (2k,2k+1)),
+//   B = the activations x' [tokens][k], K-major in shared memory with the 128-byte swizzle, loaded by
+//       TMA straight from the caller's row-major matrix (rows past M are zero-filled by the copy),
+//   D = fp32 accumulators in TMEM (128 lanes x tokens columns).
+// So the big operand is streamed exactly once, 128-bit coalesced, and never touches shared memory
+// in dequantised form.
+//
+// A CTA owns one column tile (blockIdx.x), one token tile of up to 128 tokens (blockIdx.z) and one
+// contiguous range of 128-channel groups (blockIdx.y = its rank in a thread-block cluster that
+// splits K).  Warp roles: 0 = weight-tile producer (bulk copies of whole tile blobs), 1 = activation
+// producer (TMA), 2 = MMA issuer and TMEM owner, 3..10 = dequantisation, then epilogue.  The split-K
+// partial sums are exchanged through distributed shared memory and added in rank order, so the
+// result does not depend on timing.
+//
+// Every wait is bounded: when a limit expires the CTA records ROSAQ_ERR_TIMEOUT in the context's
+// status word, stops issuing work, still joins the cluster barriers, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "rosaq_internal.cuh"
 
 namespace rosaq {
 
+namespace {
+
+constexpr int kThreads = 352;
+constexpr int kDequantThreads = 256;
+constexpr int kFirstDequantWarp = 3;
+constexpr int kWSlotBytes = kInt4CodeBytes + kScaleBytes;  // 8704: one quantized tile or a quarter fp16 tile
+constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels of an fp16 tile
+constexpr int kTmemCols = 256;
+constexpr int kMaxSplits = 8;
+
+struct TcParams {
+  const uint8_t *blob;
+  long long tile_stride;
+  int g_fp16, g_quant, bits, block_groups, d_out;
+  int M, MT;                 // tokens in the problem, tokens per CTA (multiple of 16, <= 128)
+  int S;                     // K splits = cluster size along y
+  int g_bounds[kMaxSplits + 1];
+  __half *y;
+  long long ldy;
+  const int32_t *col_map;
+  int *status;
+  long long wait_limit;
+  int NX, NW, NA;            // ring depths: activation slots, weight slots, TMEM A buffers
+};
+
+// ---------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
+          "r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t holder_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]; fp16 inputs, fp32 accumulate
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
+          taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr)
+               : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & mask) | orv
+  return r;
+}
+__device__ __forceinline__ uint32_t h2_sub_mul(uint32_t v, uint32_t sub, uint32_t mul) {
+  __half2 r = __hmul2(__hsub2(*reinterpret_cast<__half2 *>(&v), *reinterpret_cast<__half2 *>(&sub)),
+                      *reinterpret_cast<__half2 *>(&mul));
+  return *reinterpret_cast<uint32_t *>(&r);
+}
+
+// K-major, 128-byte-swizzled shared-memory operand: 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3fff) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// ---------------------------------------------------------------------------------- dequantisation
+// (code - zero) * scale in fp16, exact subtraction then one rounding: codes are spliced into the
+// mantissa of a power-of-two constant (1024, 128, 64 or 16 depending on the bit position), which
+// turns them into fp16 integers without a conversion instruction.
+struct ScaleZero {
+  uint32_t s2, z1024, z128, z64, z16;
+  __device__ __forceinline__ explicit ScaleZero(uint32_t sz) {
+    const uint32_t s = sz & 0xffffu, z = sz >> 16;
+    s2 = s | (s << 16);
+    const uint32_t zz = z | (z << 16);
+    auto add = [&](uint32_t c) {
+      __half2 r = __hadd2(*reinterpret_cast<const __half2 *>(&zz), *reinterpret_cast<const __half2 *>(&c));
+      return *reinterpret_cast<uint32_t *>(&r);
+    };
+    z1024 = add(0x64006400u);
+    z128 = add(0x58005800u);
+    z64 = add(0x54005400u);
+    z16 = add(0x4C004C00u);
+  }
+};
+
+// one word = 8 INT4 codes -> 4 fp16 pairs (k, k+1), (k+2, k+3), (k+4, k+5), (k+6, k+7)
+__device__ __forceinline__ void dequant_int4_word(uint32_t q, const ScaleZero &c, uint32_t *out) {
+  const uint32_t q8 = q >> 8;
+  out[0] = h2_sub_mul(lop_and_or(q, 0x000f000fu, 0x64006400u), c.z1024, c.s2);
+  out[1] = h2_sub_mul(lop_and_or(q, 0x00f000f0u, 0x54005400u), c.z64, c.s2);
+  out[2] = h2_sub_mul(lop_and_or(q8, 0x000f000fu, 0x64006400u), c.z1024, c.s2);
+  out[3] = h2_sub_mul(lop_and_or(q8, 0x00f000f0u, 0x54005400u), c.z64, c.s2);
+}
+
+// three words = 32 INT3 codes -> 16 fp16 pairs
+__device__ __forceinline__ void dequant_int3_set(uint32_t a, uint32_t b, uint32_t cc, const ScaleZero &c,
+                                                 uint32_t *out) {
+  const uint32_t w[3] = {a, b, cc};
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const uint32_t q = w[i], q9 = q >> 9;
+    out[5 * i + 0] = h2_sub_mul(lop_and_or(q, 0x00070007u, 0x64006400u), c.z1024, c.s2);
+    out[5 * i + 1] = h2_sub_mul(lop_and_or(q, 0x00380038u, 0x58005800u), c.z128, c.s2);
+    out[5 * i + 2] = h2_sub_mul(lop_and_or(q, 0x01c001c0u, 0x4C004C00u), c.z16, c.s2);
+    out[5 * i + 3] = h2_sub_mul(lop_and_or(q9, 0x00070007u, 0x64006400u), c.z1024, c.s2);
+    out[5 * i + 4] = h2_sub_mul(lop_and_or(q9, 0x00380038u, 0x58005800u), c.z128, c.s2);
+  }
+  const uint32_t tail = ((a >> 15) & 0x00010001u) | ((b >> 14) & 0x00020002u) | ((cc >> 13) & 0x00040004u);
+  out[15] = h2_sub_mul(tail | 0x64006400u, c.z1024, c.s2);
+}
+
+// ---------------------------------------------------------------------------------- the kernel
+struct Abort {
+  volatile int *flag;     // shared
+  int *status;            // global
+  long long limit;
+  __device__ __forceinline__ bool set() const { return *flag != 0; }
+  __device__ __forceinline__ void raise() const {
+    *flag = 1;
+    atomicExch(status, (int)ROSAQ_ERR_TIMEOUT);
+  }
+  // false when the wait gave up (or somebody else already did)
+  __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    for (long long it = 0; it < limit; ++it) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((it & 63) == 63 && set()) return false;
+    }
+    raise();
+    return false;
+  }
+};
+
+template <int kBits>
+__global__ void __launch_bounds__(kThreads, 2)
+linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // carve-up (the dynamic window is 1024-byte aligned by the launch code's padding)
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int MT = p.MT;
+  const uint32_t x_slot_bytes = (uint32_t)MT * 256u;
+  const uint32_t x_ring = base;
+  const uint32_t w_ring = x_ring + p.NX * x_slot_bytes;
+  const uint32_t bars = w_ring + p.NW * kWSlotBytes;          // 8-byte aligned (all sizes multiples of 16)
+  const uint32_t bar_x_full = bars, bar_x_empty = bar_x_full + 8 * p.NX;
+  const uint32_t bar_w_full = bar_x_empty + 8 * p.NX, bar_w_empty = bar_w_full + 8 * p.NW;
+  const uint32_t bar_a_full = bar_w_empty + 8 * p.NW, bar_a_empty = bar_a_full + 8 * p.NA;
+  const uint32_t bar_d_full = bar_a_empty + 8 * p.NA;
+  const uint32_t misc = bar_d_full + 8;                        // [0] TMEM base, [1] abort flag
+  uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t *misc_ptr = reinterpret_cast<volatile uint32_t *>(gen + (misc - base));
+  const uint32_t p_buf = base;                                 // fp32 partial tile, aliases the rings afterwards
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nt = blockIdx.x, split = blockIdx.y, m0 = blockIdx.z * MT;
+  const int g_begin = p.g_bounds[split], g_end = p.g_bounds[split + 1];
+  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit};
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.NX; ++i) {
+      mbar_init(bar_x_full + 8 * i, 1);
+      mbar_init(bar_x_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < p.NW; ++i) {
+      mbar_init(bar_w_full + 8 * i, 1);
+      mbar_init(bar_w_empty + 8 * i, kDequantThreads);
+    }
+    for (int i = 0; i < p.NA; ++i) {
+      mbar_init(bar_a_full + 8 * i, kDequantThreads);
+      mbar_init(bar_a_empty + 8 * i, 1);
+    }
+    mbar_init(bar_d_full, 1);
+    misc_ptr[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) tmem_alloc(misc, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc_ptr[0];
+  const uint32_t a_col0 = (MT <= 64) ? 64u : 128u;             // A buffers follow the accumulator columns
+
+  const uint8_t *tile_base = p.blob + (long long)nt * p.tile_stride;
+  const int qbytes = quant_tile_bytes(kBits);
+
+  if (warp == 0) {
+    // ---------------- weight-tile producer
+    if (lane == 0) {
+      int uc = 0;
+      for (int g = g_begin; g < g_end && !ab.set(); ++g) {
+        const bool f16 = g < p.g_fp16;
+        const uint8_t *src = tile_base + (f16 ? (long long)g * kFp16TileBytes
+                                              : (long long)p.g_fp16 * kFp16TileBytes + (long long)(g - p.g_fp16) * qbytes);
+        const int nsub = f16 ? 4 : 1;
+        const uint32_t bytes = f16 ? kFp16SubBytes : qbytes;
+        for (int sub = 0; sub < nsub; ++sub, ++uc) {
+          const int slot = uc % p.NW;
+          if (!ab.wait(bar_w_empty + 8 * slot, ((uc / p.NW) & 1) ^ 1)) break;
+          mbar_arrive_expect_tx(bar_w_full + 8 * slot, bytes);
+          bulk_copy_g2s(w_ring + slot * kWSlotBytes, src + (long long)sub * kFp16SubBytes, bytes, bar_w_full + 8 * slot);
+        }
+      }
+      if (ab.set()) {  // let copies already in flight land before the CTA goes away
+        for (int back = 1; back <= p.NW && back <= uc; ++back) {
+          const int u = uc - back;
+          for (long long it = 0; it < p.wait_limit; ++it)
+            if (mbar_try_wait(bar_w_full + 8 * (u % p.NW), (u / p.NW) & 1)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- activation producer
+    if (lane == 0) {
+      int gc = 0;
+      for (int g = g_begin; g < g_end && !ab.set(); ++g, ++gc) {
+        const int slot = gc % p.NX;
+        if (!ab.wait(bar_x_empty + 8 * slot, ((gc / p.NX) & 1) ^ 1)) break;
+        int k0 = g * kGroup;
+        if (p.block_groups > 0) k0 = ((nt / p.block_groups) * p.block_groups + g) * kGroup;
+        mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
+        tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
+        tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
+      }
+      if (ab.set()) {
+        for (int back = 1; back <= p.NX && back <= gc; ++back) {
+          const int u = gc - back;
+          for (long long it = 0; it < p.wait_limit; ++it)
+            if (mbar_try_wait(bar_x_full + 8 * (u % p.NX), (u / p.NX) & 1)) break;
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
+      int uc = 0, gc = 0;
+      uint32_t accumulate = 0;
+      bool ok = true;
+      for (int g = g_begin; g < g_end && ok; ++g, ++gc) {
+        const int xs = gc % p.NX;
+        if (!ab.wait(bar_x_full + 8 * xs, (gc / p.NX) & 1)) break;
+        const bool f16 = g < p.g_fp16;
+        const int nsub = f16 ? 4 : 1, ksteps = f16 ? 2 : 8;
+        for (int sub = 0; sub < nsub; ++sub, ++uc) {
+          const int ai = uc % p.NA;
+          if (!ab.wait(bar_a_full + 8 * ai, (uc / p.NA) & 1)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          for (int ks = 0; ks < ksteps; ++ks) {
+            const int koff = (f16 ? sub * 32 : 0) + ks * 16;
+            const uint32_t b_addr = x_ring + xs * x_slot_bytes + (koff >> 6) * (MT * 128) + (koff & 63) * 2;
+            tc_mma_ts(tmem, tmem + a_col0 + ai * 64 + ks * 8, make_b_desc(b_addr), idesc, accumulate);
+            accumulate = 1;
+          }
+          tc_commit(bar_a_empty + 8 * ai);
+        }
+        if (ok) tc_commit(bar_x_empty + 8 * xs);
+      }
+      tc_commit(bar_d_full);
+    }
+  } else {
+    // ---------------- dequantisation warps: shared memory -> registers -> TMEM
+    const int dq = warp - kFirstDequantWarp;       // 0..7
+    const int quad = warp & 3;                     // TMEM lane quadrant this warp may touch
+    const int hf = dq >> 2;                        // which half of the unit's K range
+    const int n = quad * 32 + lane;                // output column inside the tile = TMEM lane
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    int uc = 0;
+    bool ok = true;
+    for (int g = g_begin; g < g_end && ok; ++g) {
+      const bool f16 = g < p.g_fp16;
+      const int nsub = f16 ? 4 : 1;
+      for (int sub = 0; sub < nsub; ++sub, ++uc) {
+        const int slot = uc % p.NW, ai = uc % p.NA;
+        bool got = ab.wait(bar_w_full + 8 * slot, (uc / p.NW) & 1) &&
+                   ab.wait(bar_a_empty + 8 * ai, ((uc / p.NA) & 1) ^ 1);
+        got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
+        if (!got) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t ws = w_ring + slot * kWSlotBytes;
+        const uint32_t a_addr = lane_addr + a_col0 + ai * 64;
+        if (f16) {
+          uint32_t r[8];
+          *reinterpret_cast<uint4 *>(&r[0]) = lds128(ws + ((2 * hf + 0) * kTileN + n) * 16);
+          *reinterpret_cast<uint4 *>(&r[4]) = lds128(ws + ((2 * hf + 1) * kTileN + n) * 16);
+          tmem_st8(a_addr + 8 * hf, r);
+        } else if (kBits == 4) {
+          const ScaleZero c(lds32(ws + kInt4CodeBytes + n * 4));
+          uint32_t r[32];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint4 q = lds128(ws + ((2 * hf + j) * kTileN + n) * 16);
+            dequant_int4_word(q.x, c, &r[16 * j + 0]);
+            dequant_int4_word(q.y, c, &r[16 * j + 4]);
+            dequant_int4_word(q.z, c, &r[16 * j + 8]);
+            dequant_int4_word(q.w, c, &r[16 * j + 12]);
+          }
+          tmem_st16(a_addr + 32 * hf, &r[0]);
+          tmem_st16(a_addr + 32 * hf + 16, &r[16]);
+        } else {
+          const ScaleZero c(lds32(ws + kInt3CodeBytes + n * 4));
+          // this half needs words 6*hf .. 6*hf+5 of the column's 12: chunks hf and hf+1
+          const uint4 qa = lds128(ws + ((hf + 0) * kTileN + n) * 16);
+          const uint4 qb = lds128(ws + ((hf + 1) * kTileN + n) * 16);
+          uint32_t w6[6];
+          if (hf == 0) {
+            w6[0] = qa.x, w6[1] = qa.y, w6[2] = qa.z, w6[3] = qa.w, w6[4] = qb.x, w6[5] = qb.y;
+          } else {
+            w6[0] = qa.z, w6[1] = qa.w, w6[2] = qb.x, w6[3] = qb.y, w6[4] = qb.z, w6[5] = qb.w;
+          }
+          uint32_t r[32];
+          dequant_int3_set(w6[0], w6[1], w6[2], c, &r[0]);
+          dequant_int3_set(w6[3], w6[4], w6[5], c, &r[16]);
+          tmem_st16(a_addr + 32 * hf, &r[0]);
+          tmem_st16(a_addr + 32 * hf + 16, &r[16]);
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_a_full + 8 * ai);
+        mbar_arrive(bar_w_empty + 8 * slot);
+      }
+    }
+    // ---------------- epilogue part 1: accumulators -> fp32 partial tile in shared memory
+    bool have_d = ok && ab.wait(bar_d_full, 0);
+    have_d = __all_sync(0xffffffffu, have_d);
+    if (have_d) {
+      tc_fence_after();
+      const int half_cols = MT >> 1;               // this warp's share of the token columns
+      for (int c0 = 0; c0 < half_cols; c0 += 8) {
+        uint32_t v[8];
+        const int col = hf * half_cols + c0;
+        tmem_ld8(lane_addr + col, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          *reinterpret_cast<uint32_t *>(gen + (p_buf - base) + ((col + e) * kTileN + n) * 4) = v[e];
+      }
+    }
+  }
+
+  // ---------------- epilogue part 2: split-K sum over the cluster in rank order, fp16 store
+  tc_fence_before();
+  __syncthreads();
+  if (p.S > 1) cluster_sync_all();
+  if (warp >= kFirstDequantWarp && !ab.set()) {
+    const int tid = threadIdx.x - kFirstDequantWarp * 32;
+    const uint32_t rank = p.S > 1 ? cluster_rank() : 0;
+    const int rows = (MT - (int)rank + p.S - 1) / p.S;    // token rows rank, rank+S, ...
+    const int n0 = nt * kTileN;
+    for (int it = tid; it < rows * 32; it += kDequantThreads) {
+      const int m = (int)rank + (it >> 5) * p.S, i4 = it & 31;
+      const uint32_t off = p_buf + (uint32_t)(m * kTileN + i4 * 4) * 4;
+      float4 acc;
+      if (p.S > 1) {
+        acc = ld_cluster_f4(map_to_rank(off, 0));
+        for (int s = 1; s < p.S; ++s) {
+          const float4 v = ld_cluster_f4(map_to_rank(off, s));
+          acc.x += v.x, acc.y += v.y, acc.z += v.z, acc.w += v.w;
+        }
+      } else {
+        acc = *reinterpret_cast<const float4 *>(gen + (off - base));
+      }
+      const int mg = m0 + m, n = n0 + i4 * 4;
+      if (mg >= p.M || n >= p.d_out) continue;
+      __align__(8) __half h[4] = {__float2half_rn(acc.x), __float2half_rn(acc.y), __float2half_rn(acc.z), __float2half_rn(acc.w)};
+      __half *row = p.y + (long long)mg * p.ldy;
+      if (!p.col_map && n + 3 < p.d_out) {
+        *reinterpret_cast<uint2 *>(row + n) = *reinterpret_cast<const uint2 *>(h);
+      } else {
+        for (int e = 0; e < 4 && n + e < p.d_out; ++e) row[p.col_map ? p.col_map[n + e] : n + e] = h[e];
+      }
+    }
+  }
+  if (p.S > 1) cluster_sync_all();   // nobody leaves while a peer may still read its partial tile
+  __syncthreads();
+  if (warp == 2) {
+    __syncwarp();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+    else
+      (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+size_t smem_bytes(int MT, int NX, int NW, int NA) {
+  return 1024 + (size_t)NX * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NX + 2 * NW + 2 * NA + 1) + 16;
+}
+
+}  // namespace
+
+int tc_env_int(const char *name, int dflt) {
+  const char *v = getenv(name);
+  return v && *v ? atoi(v) : dflt;
+}
+
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
                      const int32_t *col_map, __half *y, long long ldy, cudaStream_t s) {
-  return launch_linear_simt(ctx, x, M, ldx, t, col_map, y, ldy, s);
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return ROSAQ_ERR_CUDA;
+  const int G = groups_per_tile(t);
+  if (G <= 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+
+  TcParams p{};
+  p.blob = t.blob;
+  p.tile_stride = t.tile_stride;
+  p.g_fp16 = t.g_fp16;
+  p.g_quant = t.g_quant;
+  p.bits = t.bits;
+  p.block_groups = t.block_groups;
+  p.d_out = t.d_out;
+  p.M = M;
+  const int m_tiles = (M + 127) / 128;
+  const int per_tile = (M + m_tiles - 1) / m_tiles;
+  p.MT = ((per_tile + 15) / 16) * 16;
+  p.y = y;
+  p.ldy = ldy;
+  p.col_map = col_map;
+  p.status = ctx->d_status;
+  p.wait_limit = ctx->wait_limit;
+  if (p.MT <= 64) {
+    p.NX = 2, p.NW = 9, p.NA = 3;
+  } else {
+    p.NX = 2, p.NW = 5, p.NA = 2;
+  }
+
+  // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
+  // equal bytes (an fp16 group weighs four quantized ones)
+  const int tiles = t.n_tiles * m_tiles;
+  int S = (2 * ctx->sm_count) / (tiles > 0 ? tiles : 1);
+  S = S < 1 ? 1 : (S > kMaxSplits ? kMaxSplits : S);
+  if (S > G) S = G;
+  const int forced = tc_env_int("ROSAQ_TC_SPLITS", 0);
+  if (forced >= 1 && forced <= kMaxSplits && forced <= G) S = forced;
+  p.S = S;
+  {
+    // cost(g) = 4 for an fp16 group, 1 for a quantized one; bound sp is the first group whose
+    // preceding cost reaches sp/S of the total, clamped so that every range keeps a group
+    auto cost_before = [&](int g) { return g <= t.g_fp16 ? 4ll * g : 4ll * t.g_fp16 + (g - t.g_fp16); };
+    const long long total = cost_before(G);
+    p.g_bounds[0] = 0;
+    for (int sp = 1; sp < S; ++sp) {
+      int g = p.g_bounds[sp - 1] + 1;
+      while (g < G - (S - sp) && cost_before(g) * S < total * sp) ++g;
+      p.g_bounds[sp] = g;
+    }
+    p.g_bounds[S] = G;
+  }
+
+  CUtensorMap xmap;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)t.d_in, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)p.MT};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(x), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
+  }
+
+  const size_t smem = smem_bytes(p.MT, p.NX, p.NW, p.NA);
+  auto kern = (t.g_quant > 0 && t.bits == 3) ? linear_tc_kernel<3> : linear_tc_kernel<4>;
+  static bool attr_done[2] = {false, false};
+  const int ki = (t.g_quant > 0 && t.bits == 3) ? 1 : 0;
+  if (!attr_done[ki]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 115 * 1024) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return ROSAQ_ERR_CUDA;
+    }
+    attr_done[ki] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(t.n_tiles, S, m_tiles);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = S;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = S > 1 ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, xmap, p);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
+  return ROSAQ_OK;
 }
 
 }  // namespace rosaq

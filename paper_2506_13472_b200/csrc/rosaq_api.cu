@@ -107,7 +107,7 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->sm_count = prop.multiProcessorCount;
   ctx->ws = nullptr;
   ctx->ws_bytes = 0;
-  ctx->wait_limit = 1ll << 26;
+  ctx->wait_limit = 1ll << 20;
   ctx->impl = 0;
   st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), sizeof(int)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
