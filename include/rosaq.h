@@ -177,6 +177,31 @@ int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
 int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r,
                  const rosaq_weight *w, void *y, int64_t ldy, void *stream);
 
+/*
+ * Same result as rosaq_linear, for callers that cannot allocate device memory.  (The paper has
+ * no counterpart; this entry point exists for deployment reasons only.)
+ *
+ * rosaq_linear keeps the rotated activations x . R in a context workspace that it grows with
+ * cudaMalloc on demand.  A process whose memory pool already owns all free device memory, a
+ * latency-critical loop that cannot take the device-wide synchronisation of an allocation, or a
+ * host framework that forbids allocations outside its own allocator cannot use that.  This
+ * variant keeps x . R in a fixed 4 MiB array inside the library image instead (every GPU that
+ * loads the library holds those 4 MiB until the process exits) and calls neither cudaMalloc nor
+ * cudaFree nor any allocating routine.  Inputs and outputs are still the caller's buffers.
+ *   - Limit: with r != NULL, M * d_in * 2 bytes must fit in 4 MiB (for example 512 tokens at
+ *     d_in = 4096); larger calls return ROSAQ_ERR_UNSUPPORTED_SHAPE and launch nothing.  With
+ *     r == NULL no scratch is needed and there is no limit.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device made current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.
+ *     Nothing in it has to start at zero: each call overwrites the [M][d_in] region it then
+ *     reads.  Two calls that may overlap on the GPU (different streams, or several host threads)
+ *     race on it and corrupt each other; serialise them on one stream.
+ * Arguments, alignment rules and status codes otherwise as rosaq_linear.
+ */
+int rosaq_linear_static(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r,
+                        const rosaq_weight *w, void *y, int64_t ldy, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

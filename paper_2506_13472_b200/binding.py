@@ -21,7 +21,7 @@ EXPORTS = [
     "rosaq_create", "rosaq_destroy", "rosaq_strerror", "rosaq_last_status", "rosaq_set_wait_limit",
     "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_weight_export",
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
-    "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear",
+    "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_static",
 ]
 
 
@@ -69,6 +69,7 @@ def lib():
                                    C.c_void_p]
         L.rosaq_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_void_p]
+        L.rosaq_linear_static.argtypes = L.rosaq_linear.argtypes
         _lib = L
     return _lib
 
@@ -189,6 +190,18 @@ class Context:
                                   _stream(stream)), "rosaq_linear")
         return out
 
+    def linear_static(self, x, weight, rotation=None, out=None, stream=None):
+        """rosaq_linear_static: same result as `linear`, but the library allocates nothing (the rotated
+        activations live in a fixed 4 MiB array inside the library).  Pass `out`: with out=None this
+        wrapper itself asks torch for the output tensor, which a caller that cannot allocate would not do."""
+        assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1
+        if out is None:
+            out = torch.empty((x.shape[0], weight.d_out), dtype=torch.float16, device=x.device)
+        _check(lib().rosaq_linear_static(self._h, _ptr(x), x.shape[0], x.stride(0),
+                                         None if rotation is None else rotation._h, weight._h, _ptr(out),
+                                         out.stride(0), _stream(stream)), "rosaq_linear_static")
+        return out
+
 
 class Weight:
     """rosaq_weight wrapper."""
@@ -287,6 +300,10 @@ def rosaq_rotate(ctx, x, rotation, out=None, stream=None):
 
 def rosaq_linear(ctx, x, weight, rotation=None, out=None, stream=None):
     return ctx.linear(x, weight, rotation, out, stream)
+
+
+def rosaq_linear_static(ctx, x, weight, rotation=None, out=None, stream=None):
+    return ctx.linear_static(x, weight, rotation, out, stream)
 
 
 def rosaq_last_status(ctx, stream=None):
