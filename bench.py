@@ -230,6 +230,35 @@ def gemm_stage_table(ctx, model, bits, peaks, reps=20):
     return out
 
 
+def profile_shape(args):
+    """One GEMM-stage shape over distinct random weight copies (>= 2 x L2), replayed from a CUDA graph:
+    the small, self-contained case that ncu captures are taken on.  Prints one line."""
+    import torch
+    from paper_2506_13472_b200 import binding as rb
+    d_in, d_out, M, bits = args.profile_shape
+    ctx = rb.Context(0)
+    g = torch.Generator(device="cuda").manual_seed(0)
+    nq = d_in - K_SALIENT
+    nw = nq // 8 if bits == 4 else nq // 32 * 3
+    qw = torch.randint(-2 ** 31, 2 ** 31 - 1, (nw, d_out), dtype=torch.int64, device="cuda", generator=g).to(torch.int32)
+    sc = (torch.rand((nq // 128, d_out), device="cuda", generator=g) * 0.01 + 0.001).half()
+    zr = torch.randint(0, 2 ** bits, (nq // 128, d_out), device="cuda", generator=g).half()
+    sal = (torch.randn((K_SALIENT, d_out), device="cuda", generator=g) * 0.02).half()
+    w0 = ctx.weight_import(d_in, d_out, bits, 128, K_SALIENT, qw, sc, zr, sal)
+    copies = args.copies or max(2, int(np.ceil(2 * 126e6 / w0.device_bytes)))
+    ws = [w0] + [ctx.weight_import(d_in, d_out, bits, 128, K_SALIENT, qw, sc, zr, sal) for _ in range(copies - 1)]
+    x = torch.randn((M, d_in), device="cuda", generator=g).half()
+    y = torch.empty((M, d_out), dtype=torch.float16, device="cuda")
+    gph = capture(lambda: [ctx.linear(x, w, None, out=y) for w in ws])
+    ts = sorted(time_graphs([gph], 1, 1) * 1e3 / copies for _ in range(args.steps))
+    us = ts[len(ts) // 2]
+    nb = gemm_bytes(d_in, d_out, M, bits)
+    assert ctx.last_status() == 0
+    print(json.dumps({"shape": f"{d_in}x{d_out}", "M": M, "bits": bits, "copies": copies, "us": round(us, 3),
+                      "us_min": round(ts[0], 3), "gbs": round(nb / us / 1e3, 1),
+                      "tflops": round(2.0 * M * d_in * d_out / us / 1e6, 1)}))
+
+
 # ----------------------------------------------------------------------------- oracle legs
 def oracle_sample(bits, seconds_hint=15.0):
     """Times the CPU oracle's forward (fp64, dequantise on the fly) on a column sample of the
@@ -370,8 +399,14 @@ def main():
     ap.add_argument("--bits", type=int, default=4, choices=[3, 4])
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape GEMM-stage / cuBLAS table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-shape", type=int, nargs=4, metavar=("D_IN", "D_OUT", "M", "BITS"),
+                    help="time the GEMM stage alone on one shape (random weights) and exit")
+    ap.add_argument("--copies", type=int, default=0, help="--profile-shape: distinct weight copies (default: 2 x L2)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.profile_shape:
+        args.steps = min(args.steps, 30)
+        return profile_shape(args)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -101,13 +101,35 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem desc]; fp16 inputs, fp32 accumulate
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] * B[smem desc]; fp16 inputs, fp32 accumulate.  The MMAs of one unit are
+// emitted as one block of back-to-back instructions sharing their predicates: issued one by one from
+// separate statements they cost the issuing thread about 100 cycles each, in a block about 45.
+// A advances by 8 TMEM columns (16 input channels) per MMA; B by 32 bytes inside a 64-channel
+// swizzle row (descriptor address field + 2), b_hi is the descriptor of the second 64-channel half.
+__device__ __forceinline__ void tc_mma8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_lo, uint64_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, p;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 16;\n\tadd.u64 t, %2, 4;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 24;\n\tadd.u64 t, %2, 6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 32;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], %3, %4, q;\n\t"
+      "add.u32 a, %1, 40;\n\tadd.u64 t, %3, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 48;\n\tadd.u64 t, %3, 4;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 56;\n\tadd.u64 t, %3, 6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the two MMAs of a 32-channel slice of an fp16 group
+__device__ __forceinline__ void tc_mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %3, q;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -236,12 +258,26 @@ struct Abort {
   }
   // false when the wait gave up (or somebody else already did)
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    if (mbar_try_wait(bar, parity)) return true;
     for (long long it = 0; it < limit; ++it) {
       if (mbar_try_wait(bar, parity)) return true;
       if ((it & 63) == 63 && set()) return false;
     }
     raise();
     return false;
+  }
+};
+
+// Position in a ring of n slots plus the parity of the current lap, advanced without division
+// (the role warps run on a single lane: an integer division there costs hundreds of cycles).
+struct Ring {
+  int idx;
+  uint32_t lap;
+  __device__ __forceinline__ void advance(int n) {
+    if (++idx == n) {
+      idx = 0;
+      lap ^= 1u;
+    }
   }
 };
 
@@ -302,15 +338,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     // ---------------- weight-tile producer
     if (lane == 0) {
       int uc = 0;
+      Ring rw{0, 0};
       for (int g = g_begin; g < g_end && !ab.set(); ++g) {
         const bool f16 = g < p.g_fp16;
         const uint8_t *src = tile_base + (f16 ? (long long)g * kFp16TileBytes
                                               : (long long)p.g_fp16 * kFp16TileBytes + (long long)(g - p.g_fp16) * qbytes);
         const int nsub = f16 ? 4 : 1;
         const uint32_t bytes = f16 ? kFp16SubBytes : qbytes;
-        for (int sub = 0; sub < nsub; ++sub, ++uc) {
-          const int slot = uc % p.NW;
-          if (!ab.wait(bar_w_empty + 8 * slot, ((uc / p.NW) & 1) ^ 1)) break;
+        for (int sub = 0; sub < nsub; ++sub, ++uc, rw.advance(p.NW)) {
+          const int slot = rw.idx;
+          if (!ab.wait(bar_w_empty + 8 * slot, rw.lap ^ 1u)) break;
           mbar_arrive_expect_tx(bar_w_full + 8 * slot, bytes);
           bulk_copy_g2s(w_ring + slot * kWSlotBytes, src + (long long)sub * kFp16SubBytes, bytes, bar_w_full + 8 * slot);
         }
@@ -327,11 +364,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     // ---------------- activation producer
     if (lane == 0) {
       int gc = 0;
-      for (int g = g_begin; g < g_end && !ab.set(); ++g, ++gc) {
-        const int slot = gc % p.NX;
-        if (!ab.wait(bar_x_empty + 8 * slot, ((gc / p.NX) & 1) ^ 1)) break;
-        int k0 = g * kGroup;
-        if (p.block_groups > 0) k0 = ((nt / p.block_groups) * p.block_groups + g) * kGroup;
+      Ring rx{0, 0};
+      // block-diagonal operand: column tile nt only multiplies the channels of its own diagonal block
+      const int g_block0 = p.block_groups > 0 ? (nt / p.block_groups) * p.block_groups : 0;
+      for (int g = g_begin; g < g_end && !ab.set(); ++g, ++gc, rx.advance(p.NX)) {
+        const int slot = rx.idx;
+        if (!ab.wait(bar_x_empty + 8 * slot, rx.lap ^ 1u)) break;
+        const int k0 = (g_block0 + g) * kGroup;
         mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
         tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
         tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
@@ -348,27 +387,30 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     // ---------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
-      int uc = 0, gc = 0;
+      const uint64_t desc0 = make_b_desc(x_ring);            // descriptor address fields are in 16-byte units
+      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MT * 128) >> 4;
+      Ring rx{0, 0}, ra{0, 0};
       uint32_t accumulate = 0;
       bool ok = true;
-      for (int g = g_begin; g < g_end && ok; ++g, ++gc) {
-        const int xs = gc % p.NX;
-        if (!ab.wait(bar_x_full + 8 * xs, (gc / p.NX) & 1)) break;
+      for (int g = g_begin; g < g_end && ok; ++g, rx.advance(p.NX)) {
+        const int xs = rx.idx;
+        if (!ab.wait(bar_x_full + 8 * xs, rx.lap)) break;
         const bool f16 = g < p.g_fp16;
-        const int nsub = f16 ? 4 : 1, ksteps = f16 ? 2 : 8;
-        for (int sub = 0; sub < nsub; ++sub, ++uc) {
-          const int ai = uc % p.NA;
-          if (!ab.wait(bar_a_full + 8 * ai, (uc / p.NA) & 1)) {
+        const int nsub = f16 ? 4 : 1;
+        for (int sub = 0; sub < nsub; ++sub, ra.advance(p.NA)) {
+          const int ai = ra.idx;
+          if (!ab.wait(bar_a_full + 8 * ai, ra.lap)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const int koff = (f16 ? sub * 32 : 0) + ks * 16;
-            const uint32_t b_addr = x_ring + xs * x_slot_bytes + (koff >> 6) * (MT * 128) + (koff & 63) * 2;
-            tc_mma_ts(tmem, tmem + a_col0 + ai * 64 + ks * 8, make_b_desc(b_addr), idesc, accumulate);
-            accumulate = 1;
-          }
+          const uint32_t a_tmem = tmem + a_col0 + ai * 64;
+          const uint64_t b0 = desc0 + (uint64_t)(xs * x_slot16);
+          if (f16)
+            tc_mma2_ts(tmem, a_tmem, b0 + (uint64_t)((sub >> 1) * half16 + (sub & 1) * 4), idesc, accumulate);
+          else
+            tc_mma8_ts(tmem, a_tmem, b0, b0 + (uint64_t)half16, idesc, accumulate);
+          accumulate = 1;
           tc_commit(bar_a_empty + 8 * ai);
         }
         if (ok) tc_commit(bar_x_empty + 8 * xs);
@@ -382,15 +424,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     const int hf = dq >> 2;                        // which half of the unit's K range
     const int n = quad * 32 + lane;                // output column inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    int uc = 0;
+    Ring rw{0, 0}, ra{0, 0};
     bool ok = true;
     for (int g = g_begin; g < g_end && ok; ++g) {
       const bool f16 = g < p.g_fp16;
       const int nsub = f16 ? 4 : 1;
-      for (int sub = 0; sub < nsub; ++sub, ++uc) {
-        const int slot = uc % p.NW, ai = uc % p.NA;
-        bool got = ab.wait(bar_w_full + 8 * slot, (uc / p.NW) & 1) &&
-                   ab.wait(bar_a_empty + 8 * ai, ((uc / p.NA) & 1) ^ 1);
+      for (int sub = 0; sub < nsub; ++sub, rw.advance(p.NW), ra.advance(p.NA)) {
+        const int slot = rw.idx, ai = ra.idx;
+        bool got = ab.wait(bar_w_full + 8 * slot, rw.lap) && ab.wait(bar_a_empty + 8 * ai, ra.lap ^ 1u);
         got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
         if (!got) {
           ok = false;
@@ -556,7 +597,11 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
   if (p.MT <= 64) {
-    p.NX = 2, p.NW = 9, p.NA = 3;
+    // activation slots are MT * 256 bytes; keep about 64 KB of them in flight so that a slot's reload
+    // (an L2 round trip of a microsecond or so) is hidden behind several groups of work
+    p.NX = 65536 / (p.MT * 256);
+    p.NX = p.NX > 8 ? 8 : p.NX;
+    p.NX = tc_env_int("ROSAQ_TC_NX", p.NX), p.NW = tc_env_int("ROSAQ_TC_NW", 5), p.NA = 3;
   } else {
     p.NX = 2, p.NW = 5, p.NA = 2;
   }
