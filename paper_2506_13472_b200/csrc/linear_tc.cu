@@ -21,6 +21,7 @@
 // Every wait is bounded: when a limit expires the CTA records ROSAQ_ERR_TIMEOUT in the context's
 // status word, stops issuing work, still joins the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
+#include <cstdio>
 
 #include "rosaq_internal.cuh"
 
@@ -48,7 +49,7 @@ struct TcParams {
   const int32_t *col_map;
   int *status;
   long long wait_limit;
-  int NX, NW, NA;            // ring depths: activation slots, weight slots, TMEM A buffers
+  int NW, NA;                // ring depths: packed-weight slots, stages (TMEM A buffer + activation slot)
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -86,13 +87,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
-__device__ __forceinline__ void tmem_alloc(uint32_t holder_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(cols)
+// The column count is an immediate on purpose: with a register operand the tools cannot see how much
+// tensor memory a CTA takes and assume all 512 columns, which limits the kernel to one CTA per SM.
+template <uint32_t kCols>
+__device__ __forceinline__ void tmem_alloc(uint32_t holder_smem) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "n"(kCols)
                : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+template <uint32_t kCols>
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "n"(kCols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -152,6 +157,8 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
                : "r"(taddr)
                : "memory");
 }
+__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -289,13 +296,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int MT = p.MT;
   const uint32_t x_slot_bytes = (uint32_t)MT * 256u;
-  const uint32_t x_ring = base;
-  const uint32_t w_ring = x_ring + p.NX * x_slot_bytes;
+  const uint32_t x_ring = base;                                // NA slots: one per TMEM operand buffer
+  const uint32_t w_ring = x_ring + p.NA * x_slot_bytes;
   const uint32_t bars = w_ring + p.NW * kWSlotBytes;          // 8-byte aligned (all sizes multiples of 16)
-  const uint32_t bar_x_full = bars, bar_x_empty = bar_x_full + 8 * p.NX;
-  const uint32_t bar_w_full = bar_x_empty + 8 * p.NX, bar_w_empty = bar_w_full + 8 * p.NW;
-  const uint32_t bar_a_full = bar_w_empty + 8 * p.NW, bar_a_empty = bar_a_full + 8 * p.NA;
-  const uint32_t bar_d_full = bar_a_empty + 8 * p.NA;
+  const uint32_t bar_w_full = bars, bar_w_empty = bar_w_full + 8 * p.NW;
+  const uint32_t bar_x_full = bar_w_empty + 8 * p.NW, bar_a_full = bar_x_full + 8 * p.NA;
+  const uint32_t bar_empty = bar_a_full + 8 * p.NA;           // stage (operand buffer + activation slot) free again
+  const uint32_t bar_d_full = bar_empty + 8 * p.NA;
   const uint32_t misc = bar_d_full + 8;                        // [0] TMEM base, [1] abort flag
   uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t *misc_ptr = reinterpret_cast<volatile uint32_t *>(gen + (misc - base));
@@ -306,25 +313,26 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const int g_begin = p.g_bounds[split], g_end = p.g_bounds[split + 1];
   const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit};
 
+  // Let the next kernel of the stream start its own prologue and weight prefetch while this one runs
+  // (it only matters when the launches are chained programmatically; otherwise a no-op).
+  grid_dep_launch_dependents();
+
   if (threadIdx.x == 0) {
-    for (int i = 0; i < p.NX; ++i) {
-      mbar_init(bar_x_full + 8 * i, 1);
-      mbar_init(bar_x_empty + 8 * i, 1);
-    }
     for (int i = 0; i < p.NW; ++i) {
       mbar_init(bar_w_full + 8 * i, 1);
       mbar_init(bar_w_empty + 8 * i, kDequantThreads);
     }
     for (int i = 0; i < p.NA; ++i) {
+      mbar_init(bar_x_full + 8 * i, 1);
       mbar_init(bar_a_full + 8 * i, kDequantThreads);
-      mbar_init(bar_a_empty + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_d_full, 1);
     misc_ptr[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 2) tmem_alloc(misc, kTmemCols);
+  if (warp == 2) tmem_alloc<kTmemCols>(misc);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -335,7 +343,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const int qbytes = quant_tile_bytes(kBits);
 
   if (warp == 0) {
-    // ---------------- weight-tile producer
+    // ---------------- weight-tile producer (weights never depend on the previous kernel: no grid wait)
     if (lane == 0) {
       int uc = 0;
       Ring rw{0, 0};
@@ -363,57 +371,43 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   } else if (warp == 1) {
     // ---------------- activation producer
     if (lane == 0) {
+      grid_dep_wait();                                         // x may be the previous kernel's output
       int gc = 0;
-      Ring rx{0, 0};
+      Ring rs{0, 0};
       // block-diagonal operand: column tile nt only multiplies the channels of its own diagonal block
       const int g_block0 = p.block_groups > 0 ? (nt / p.block_groups) * p.block_groups : 0;
-      for (int g = g_begin; g < g_end && !ab.set(); ++g, ++gc, rx.advance(p.NX)) {
-        const int slot = rx.idx;
-        if (!ab.wait(bar_x_empty + 8 * slot, rx.lap ^ 1u)) break;
+      for (int g = g_begin; g < g_end && !ab.set(); ++g, ++gc, rs.advance(p.NA)) {
+        const int slot = rs.idx;
+        if (!ab.wait(bar_empty + 8 * slot, rs.lap ^ 1u)) break;
         const int k0 = (g_block0 + g) * kGroup;
         mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
         tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
         tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
       }
       if (ab.set()) {
-        for (int back = 1; back <= p.NX && back <= gc; ++back) {
+        for (int back = 1; back <= p.NA && back <= gc; ++back) {
           const int u = gc - back;
           for (long long it = 0; it < p.wait_limit; ++it)
-            if (mbar_try_wait(bar_x_full + 8 * (u % p.NX), (u / p.NX) & 1)) break;
+            if (mbar_try_wait(bar_x_full + 8 * (u % p.NA), (u / p.NA) & 1)) break;
         }
       }
     }
   } else if (warp == 2) {
-    // ---------------- MMA issuer
+    // ---------------- MMA issuer: per group one wait pair, eight MMAs, one commit
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
       const uint64_t desc0 = make_b_desc(x_ring);            // descriptor address fields are in 16-byte units
       const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MT * 128) >> 4;
-      Ring rx{0, 0}, ra{0, 0};
+      Ring rs{0, 0};
       uint32_t accumulate = 0;
-      bool ok = true;
-      for (int g = g_begin; g < g_end && ok; ++g, rx.advance(p.NX)) {
-        const int xs = rx.idx;
-        if (!ab.wait(bar_x_full + 8 * xs, rx.lap)) break;
-        const bool f16 = g < p.g_fp16;
-        const int nsub = f16 ? 4 : 1;
-        for (int sub = 0; sub < nsub; ++sub, ra.advance(p.NA)) {
-          const int ai = ra.idx;
-          if (!ab.wait(bar_a_full + 8 * ai, ra.lap)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t a_tmem = tmem + a_col0 + ai * 64;
-          const uint64_t b0 = desc0 + (uint64_t)(xs * x_slot16);
-          if (f16)
-            tc_mma2_ts(tmem, a_tmem, b0 + (uint64_t)((sub >> 1) * half16 + (sub & 1) * 4), idesc, accumulate);
-          else
-            tc_mma8_ts(tmem, a_tmem, b0, b0 + (uint64_t)half16, idesc, accumulate);
-          accumulate = 1;
-          tc_commit(bar_a_empty + 8 * ai);
-        }
-        if (ok) tc_commit(bar_x_empty + 8 * xs);
+      for (int g = g_begin; g < g_end; ++g, rs.advance(p.NA)) {
+        const int st = rs.idx;
+        if (!ab.wait(bar_x_full + 8 * st, rs.lap) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
+        tc_fence_after();
+        const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
+        tc_mma8_ts(tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+        accumulate = 1;
+        tc_commit(bar_empty + 8 * st);
       }
       tc_commit(bar_d_full);
     }
@@ -421,17 +415,20 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     // ---------------- dequantisation warps: shared memory -> registers -> TMEM
     const int dq = warp - kFirstDequantWarp;       // 0..7
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may touch
-    const int hf = dq >> 2;                        // which half of the unit's K range
+    const int hf = dq >> 2;                        // which half of the slot's K range
     const int n = quad * 32 + lane;                // output column inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    Ring rw{0, 0}, ra{0, 0};
+    Ring rw{0, 0}, rs{0, 0};
     bool ok = true;
-    for (int g = g_begin; g < g_end && ok; ++g) {
+    for (int g = g_begin; g < g_end && ok; ++g, rs.advance(p.NA)) {
       const bool f16 = g < p.g_fp16;
       const int nsub = f16 ? 4 : 1;
-      for (int sub = 0; sub < nsub; ++sub, rw.advance(p.NW), ra.advance(p.NA)) {
-        const int slot = rw.idx, ai = ra.idx;
-        bool got = ab.wait(bar_w_full + 8 * slot, rw.lap) && ab.wait(bar_a_empty + 8 * ai, ra.lap ^ 1u);
+      const int st = rs.idx;
+      const uint32_t a_addr = lane_addr + a_col0 + st * 64;
+      bool got = ab.wait(bar_empty + 8 * st, rs.lap ^ 1u);
+      for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(p.NW)) {
+        const int slot = rw.idx;
+        got = got && ab.wait(bar_w_full + 8 * slot, rw.lap);
         got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
         if (!got) {
           ok = false;
@@ -439,30 +436,35 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
         }
         tc_fence_after();
         const uint32_t ws = w_ring + slot * kWSlotBytes;
-        const uint32_t a_addr = lane_addr + a_col0 + ai * 64;
         if (f16) {
+          // a quarter of an fp16 group: 32 input channels = 16 TMEM columns, 8 per half
           uint32_t r[8];
           *reinterpret_cast<uint4 *>(&r[0]) = lds128(ws + ((2 * hf + 0) * kTileN + n) * 16);
           *reinterpret_cast<uint4 *>(&r[4]) = lds128(ws + ((2 * hf + 1) * kTileN + n) * 16);
-          tmem_st8(a_addr + 8 * hf, r);
+          mbar_arrive(bar_w_empty + 8 * slot);
+          tmem_st8(a_addr + 16 * sub + 8 * hf, r);
         } else if (kBits == 4) {
           const ScaleZero c(lds32(ws + kInt4CodeBytes + n * 4));
+          const uint4 q0 = lds128(ws + ((2 * hf + 0) * kTileN + n) * 16);
+          const uint4 q1 = lds128(ws + ((2 * hf + 1) * kTileN + n) * 16);
+          mbar_arrive(bar_w_empty + 8 * slot);
           uint32_t r[32];
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const uint4 q = lds128(ws + ((2 * hf + j) * kTileN + n) * 16);
-            dequant_int4_word(q.x, c, &r[16 * j + 0]);
-            dequant_int4_word(q.y, c, &r[16 * j + 4]);
-            dequant_int4_word(q.z, c, &r[16 * j + 8]);
-            dequant_int4_word(q.w, c, &r[16 * j + 12]);
-          }
+          dequant_int4_word(q0.x, c, &r[0]);
+          dequant_int4_word(q0.y, c, &r[4]);
+          dequant_int4_word(q0.z, c, &r[8]);
+          dequant_int4_word(q0.w, c, &r[12]);
           tmem_st16(a_addr + 32 * hf, &r[0]);
+          dequant_int4_word(q1.x, c, &r[16]);
+          dequant_int4_word(q1.y, c, &r[20]);
+          dequant_int4_word(q1.z, c, &r[24]);
+          dequant_int4_word(q1.w, c, &r[28]);
           tmem_st16(a_addr + 32 * hf + 16, &r[16]);
         } else {
           const ScaleZero c(lds32(ws + kInt3CodeBytes + n * 4));
           // this half needs words 6*hf .. 6*hf+5 of the column's 12: chunks hf and hf+1
           const uint4 qa = lds128(ws + ((hf + 0) * kTileN + n) * 16);
           const uint4 qb = lds128(ws + ((hf + 1) * kTileN + n) * 16);
+          mbar_arrive(bar_w_empty + 8 * slot);
           uint32_t w6[6];
           if (hf == 0) {
             w6[0] = qa.x, w6[1] = qa.y, w6[2] = qa.z, w6[3] = qa.w, w6[4] = qb.x, w6[5] = qb.y;
@@ -471,15 +473,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
           }
           uint32_t r[32];
           dequant_int3_set(w6[0], w6[1], w6[2], c, &r[0]);
-          dequant_int3_set(w6[3], w6[4], w6[5], c, &r[16]);
           tmem_st16(a_addr + 32 * hf, &r[0]);
+          dequant_int3_set(w6[3], w6[4], w6[5], c, &r[16]);
           tmem_st16(a_addr + 32 * hf + 16, &r[16]);
         }
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar_a_full + 8 * ai);
-        mbar_arrive(bar_w_empty + 8 * slot);
       }
+      if (!ok) break;
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_a_full + 8 * st);
     }
     // ---------------- epilogue part 1: accumulators -> fp32 partial tile in shared memory
     bool have_d = ok && ab.wait(bar_d_full, 0);
@@ -504,6 +506,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   __syncthreads();
   if (p.S > 1) cluster_sync_all();
   if (warp >= kFirstDequantWarp && !ab.set()) {
+    grid_dep_wait();                                         // y may still be read by the previous kernel
     const int tid = threadIdx.x - kFirstDequantWarp * 32;
     const uint32_t rank = p.S > 1 ? cluster_rank() : 0;
     const int rows = (MT - (int)rank + p.S - 1) / p.S;    // token rows rank, rank+S, ...
@@ -536,7 +539,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   __syncthreads();
   if (warp == 2) {
     __syncwarp();
-    tmem_dealloc(tmem, kTmemCols);
+    tmem_dealloc<kTmemCols>(tmem);
   }
 }
 
@@ -561,8 +564,11 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-size_t smem_bytes(int MT, int NX, int NW, int NA) {
-  return 1024 + (size_t)NX * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NX + 2 * NW + 2 * NA + 1) + 16;
+size_t smem_bytes(int MT, int NW, int NA) {
+  size_t b = 1024 + (size_t)NA * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NW + 3 * NA + 1) + 16;
+  // never less than a third of an SM's shared memory: at most two CTAs share an SM, which is also what
+  // their 2 x 256 tensor-memory columns allow
+  return b < 80 * 1024 ? 80 * 1024 : b;
 }
 
 }  // namespace
@@ -596,14 +602,13 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
   p.col_map = col_map;
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
-  if (p.MT <= 64) {
-    // activation slots are MT * 256 bytes; keep about 64 KB of them in flight so that a slot's reload
-    // (an L2 round trip of a microsecond or so) is hidden behind several groups of work
-    p.NX = 65536 / (p.MT * 256);
-    p.NX = p.NX > 8 ? 8 : p.NX;
-    p.NX = tc_env_int("ROSAQ_TC_NX", p.NX), p.NW = tc_env_int("ROSAQ_TC_NW", 5), p.NA = 3;
-  } else {
-    p.NX = 2, p.NW = 5, p.NA = 2;
+  // stages (TMEM operand buffer + activation slot of MT x 128 channels): 3 next to 64 accumulator
+  // columns, 2 next to 128; the rest of a half SM's shared memory goes to the packed-weight ring
+  p.NA = p.MT <= 64 ? 3 : 2;
+  {
+    const int budget = 110 * 1024 - 1024 - p.NA * p.MT * 256 - 256;
+    int nw = budget / kWSlotBytes;
+    p.NW = tc_env_int("ROSAQ_TC_NW", nw > 10 ? 10 : nw);
   }
 
   // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
@@ -641,29 +646,61 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
     if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
   }
 
-  const size_t smem = smem_bytes(p.MT, p.NX, p.NW, p.NA);
+  const size_t smem = smem_bytes(p.MT, p.NW, p.NA);
   auto kern = (t.g_quant > 0 && t.bits == 3) ? linear_tc_kernel<3> : linear_tc_kernel<4>;
-  static bool attr_done[2] = {false, false};
+  // The opt-in limit is kept equal to what the launches really need (never a rounder, larger figure):
+  // the driver sizes the shared-memory carve-out and the CTAs per SM from this attribute, and with
+  // 2 x (limit + 1 KB) above the SM's 228 KB only one CTA would be resident.
+  static size_t attr_smem[2] = {0, 0};
   const int ki = (t.g_quant > 0 && t.bits == 3) ? 1 : 0;
-  if (!attr_done[ki]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 115 * 1024) != cudaSuccess) {
+  if (attr_smem[ki] < smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       (void)cudaGetLastError();
       return ROSAQ_ERR_CUDA;
     }
-    attr_done[ki] = true;
+    attr_smem[ki] = smem;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(t.n_tiles, S, m_tiles);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1;
-  attr[0].val.clusterDim.y = S;
-  attr[0].val.clusterDim.z = 1;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (S > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1;
+    attr[na].val.clusterDim.y = S;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (tc_env_int("ROSAQ_TC_PDL", 1)) {
+    // programmatic dependent launch: this kernel may start while the previous kernel of the stream is
+    // still running; it touches x and y only after griddepcontrol.wait
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = S > 1 ? 1 : 0;
+  cfg.numAttrs = na;
+  if (tc_env_int("ROSAQ_TC_DEBUG", 0)) {
+    int nc = -1, nb = -1;
+    cudaOccupancyMaxActiveClusters(&nc, kern, &cfg);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, kThreads, smem);
+    cudaFuncAttributes fa;
+    cudaFuncGetAttributes(&fa, kern);
+    fprintf(stderr, "attrs: regs %d static smem %zu const %zu local %zu maxThreads %d maxDyn %d carveout %d\n", fa.numRegs,
+            fa.sharedSizeBytes, fa.constSizeBytes, fa.localSizeBytes, fa.maxThreadsPerBlock, fa.maxDynamicSharedSizeBytes,
+            fa.preferredShmemCarveout);
+    for (int kb = 40; kb <= 112; kb += 8) {
+      int n2 = -1;
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, kern, kThreads, (size_t)kb * 1024);
+      fprintf(stderr, "  dyn smem %d KB -> %d blocks/SM\n", kb, n2);
+    }
+    fprintf(stderr, "linear_tc: grid %d x %d x %d, MT %d, smem %zu, NW %d NA %d, max active clusters %d, blocks/SM %d\n",
+            t.n_tiles, S, m_tiles, p.MT, smem, p.NW, p.NA, nc, nb);
+  }
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, xmap, p);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
