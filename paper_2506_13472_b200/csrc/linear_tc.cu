@@ -21,7 +21,6 @@
 // Every wait is bounded: when a limit expires the CTA records ROSAQ_ERR_TIMEOUT in the context's
 // status word, stops issuing work, still joins the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
-#include <cstdio>
 
 #include "rosaq_internal.cuh"
 
@@ -516,11 +515,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       const uint32_t off = p_buf + (uint32_t)(m * kTileN + i4 * 4) * 4;
       float4 acc;
       if (p.S > 1) {
-        acc = ld_cluster_f4(map_to_rank(off, 0));
-        for (int s = 1; s < p.S; ++s) {
-          const float4 v = ld_cluster_f4(map_to_rank(off, s));
-          acc.x += v.x, acc.y += v.y, acc.z += v.z, acc.w += v.w;
-        }
+        // all remote loads are issued before the first add (a DSMEM round trip each); the sum still
+        // runs in rank order
+        float4 v[kMaxSplits];
+#pragma unroll
+        for (int s = 0; s < kMaxSplits; ++s)
+          v[s] = s < p.S ? ld_cluster_f4(map_to_rank(off, s)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc = v[0];
+#pragma unroll
+        for (int s = 1; s < kMaxSplits; ++s)
+          if (s < p.S) acc.x += v[s].x, acc.y += v[s].y, acc.z += v[s].z, acc.w += v[s].w;
       } else {
         acc = *reinterpret_cast<const float4 *>(gen + (off - base));
       }
@@ -684,23 +688,6 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
   }
   cfg.attrs = attr;
   cfg.numAttrs = na;
-  if (tc_env_int("ROSAQ_TC_DEBUG", 0)) {
-    int nc = -1, nb = -1;
-    cudaOccupancyMaxActiveClusters(&nc, kern, &cfg);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, kThreads, smem);
-    cudaFuncAttributes fa;
-    cudaFuncGetAttributes(&fa, kern);
-    fprintf(stderr, "attrs: regs %d static smem %zu const %zu local %zu maxThreads %d maxDyn %d carveout %d\n", fa.numRegs,
-            fa.sharedSizeBytes, fa.constSizeBytes, fa.localSizeBytes, fa.maxThreadsPerBlock, fa.maxDynamicSharedSizeBytes,
-            fa.preferredShmemCarveout);
-    for (int kb = 40; kb <= 112; kb += 8) {
-      int n2 = -1;
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, kern, kThreads, (size_t)kb * 1024);
-      fprintf(stderr, "  dyn smem %d KB -> %d blocks/SM\n", kb, n2);
-    }
-    fprintf(stderr, "linear_tc: grid %d x %d x %d, MT %d, smem %zu, NW %d NA %d, max active clusters %d, blocks/SM %d\n",
-            t.n_tiles, S, m_tiles, p.MT, smem, p.NW, p.NA, nc, nb);
-  }
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, xmap, p);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
