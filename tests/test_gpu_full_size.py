@@ -1,0 +1,114 @@
+"""GPU parity at the full benchmark sizes (LLaMA-7B and 13B shaped linears), in the launch
+configuration the benchmark times, on sampled output columns that the CPU oracle computes one by one.
+
+Integer results (codes, scales, zeros, salient bits) of the sampled columns must be bit-exact;
+y on the sampled columns must satisfy ||y - y_ref||_F / ||y_ref||_F <= 2e-3 against the oracle's fp64
+forward on the same dequantised weights.  The rotation R is an input of the calls (any orthogonal
+matrix will do for parity): a product of seeded Householder reflectors, exactly orthogonal in fp64.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rosaq_oracle as orc
+from paper_2506_13472_b200 import binding as rb
+from paper_2506_13472_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+N_COLS = 24       # sampled output columns per case (always includes 0, 127, 128 and the last one)
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = rb.Context(0)
+    yield c
+    c.close()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def householder_rotation(d, seed, key):
+    vs = synth.householder_vectors(d, 6, synth.rng_for(seed, key, "R"))
+    return synth.apply_householders(np.eye(d), vs)
+
+
+def check_case(ctx, d_in, d_out, bits, Ms, seed, key, heavy_tail=False, sigma=0.02):
+    R64 = householder_rotation(d_in, seed, key)
+    R32, R16 = R64.astype(np.float32), R64.astype(np.float16)
+    W = synth.weights(d_in, d_out, seed, key, sigma=sigma, outlier_frac=0.005 if heavy_tail else 0.01,
+                      outlier_scale=10.0, heavy_tail=heavy_tail)
+    cols = synth.sample_columns(d_out, N_COLS, seed, key)
+    w = ctx.quantize(dev(W), dev(R32), bits=bits, k_salient=128)
+    qd = H.oracle_quantized(W, R32, None, bits, 128, cols=cols)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    rot = ctx.rotation_create(dev(R16))
+    law = synth.ActivationLaw(d_in, 1.0, seed, key + "/x")
+    for M in Ms:
+        x = law.sample(M, f"x{M}", np.float16)
+        xd = dev(x)
+        xr = ctx.rotate(xd, rot)
+        y = ctx.linear(xr, w, None)                       # the GEMM stage the benchmark times
+        y_fused = ctx.linear(xd, w, rot)                  # the single-call form
+        assert ctx.last_status() == rb.ROSAQ_OK
+        y_ref, xr_ref = orc.forward(x, qd, R16, None, return_xrot=True)
+        assert H.rel_fro(xr.cpu().numpy(), xr_ref) <= 1e-3
+        got = y.cpu().numpy()
+        assert np.all(np.isfinite(got))
+        assert H.rel_fro(got[:, cols], y_ref) <= H.REL_TOL_Y
+        assert np.array_equal(y_fused.cpu().numpy().view(np.uint16), got.view(np.uint16))
+    w.free()
+    rot.free()
+
+
+@pytest.mark.parametrize("d_in,d_out", [(4096, 4096), (4096, 11008), (11008, 4096)])
+def test_7b_shapes_int4_m64(ctx, d_in, d_out):
+    check_case(ctx, d_in, d_out, 4, [64], seed=1, key=f"7b{d_in}x{d_out}")
+
+
+def test_7b_int3_m_sweep(ctx):
+    check_case(ctx, 4096, 4096, 3, [1, 16, 64, 256], seed=2, key="7b-int3")
+
+
+def test_7b_int3_wide_m64(ctx):
+    check_case(ctx, 4096, 11008, 3, [64], seed=2, key="7b-int3-wide")
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+def test_13b_shape_heavy_tail_m_sweep(ctx, bits):
+    check_case(ctx, 5120, 13824, bits, [1, 64, 512], seed=4, key=f"13b{bits}", heavy_tail=True, sigma=0.015)
+
+
+def test_13b_down_shape_int4(ctx):
+    check_case(ctx, 13824, 5120, 4, [64], seed=4, key="13b-down", heavy_tail=True, sigma=0.015)
+
+
+def test_headwise_full_size_o_proj(ctx):
+    """Config 4's o_proj: 32 heads x 128, block-diagonal R from per-head PCA of synthetic per-head
+    activations plus the global descending-eigenvalue permutation; INT4, K = 128, M = 64."""
+    heads, hd, d = 32, 128, 4096
+    law = synth.HeadwiseActivationLaw(heads, hd, 3, "hw-full")
+    X = law.sample(4096, "calib", np.float16)
+    Cg = torch.zeros((heads, hd, hd), dtype=torch.float32, device="cuda")
+    ctx.calib_cov(dev(X), Cg, heads)
+    Cb = orc.cov(X, n_blocks=heads)
+    got = Cg.cpu().numpy().astype(np.float64)
+    dg = np.sqrt(np.diagonal(Cb, axis1=-2, axis2=-1))
+    assert np.all(np.abs(got - Cb) <= 2.0 ** -24 * (4 * 64 + 8) * dg[:, :, None] * dg[:, None, :] + 1e-30)
+    lams, Vs = zip(*[orc.eigh_jacobi(Cb[h]) for h in range(heads)])
+    Rb, perm = orc.assemble_headwise_rotation(np.array(lams), np.array(Vs))
+    Rb32, Rb16 = Rb.astype(np.float32), Rb.astype(np.float16)
+    W = synth.weights(d, d, 3, "hw-full", outlier_frac=0.01)
+    cols = synth.sample_columns(d, N_COLS, 3, "hw-full")
+    w = ctx.quantize(dev(W), dev(Rb32), dev(perm), bits=4, k_salient=128)
+    qd = H.oracle_quantized(W, Rb32, perm, 4, 128, cols=cols)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    rot = ctx.rotation_create(dev(Rb16), dev(perm))
+    x = law.sample(64, "x", np.float16)
+    y = ctx.linear(dev(x), w, rot).cpu().numpy()
+    assert ctx.last_status() == rb.ROSAQ_OK
+    y_ref = orc.forward(x, qd, Rb16, perm)
+    assert H.rel_fro(y[:, cols], y_ref) <= H.REL_TOL_Y
