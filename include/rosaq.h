@@ -178,6 +178,16 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
                  const rosaq_weight *w, void *y, int64_t ldy, void *stream);
 
 /*
+ * Several linears that read the same activation (q/k/v, or gate/up: they share one rotation, Section 3.1)
+ * in one launch:  y[i] = (x . R) . W^[i]  for i < n, 1 <= n <= 4, each with the result bits rosaq_linear
+ * would give.  All w[i] must have the same d_in, bits and k_salient; d_out may differ.  w, y and ldy are
+ * HOST arrays of n entries (device pointers inside); they are read before the call returns.
+ * r as in rosaq_linear (the rotation runs once).  Errors as rosaq_linear.
+ */
+int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r, int n,
+                       const rosaq_weight *const *w, void *const *y, const int64_t *ldy, void *stream);
+
+/*
  * Same result as rosaq_linear, for callers that cannot allocate device memory.  (The paper has
  * no counterpart; this entry point exists for deployment reasons only.)
  *

@@ -21,7 +21,7 @@ EXPORTS = [
     "rosaq_create", "rosaq_destroy", "rosaq_strerror", "rosaq_last_status", "rosaq_set_wait_limit",
     "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_weight_export",
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
-    "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_static",
+    "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_multi", "rosaq_linear_static",
 ]
 
 
@@ -70,6 +70,8 @@ def lib():
         L.rosaq_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_void_p]
         L.rosaq_linear_static.argtypes = L.rosaq_linear.argtypes
+        L.rosaq_linear_multi.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_int, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -190,6 +192,20 @@ class Context:
                                   _stream(stream)), "rosaq_linear")
         return out
 
+    def linear_multi(self, x, weights, rotation=None, outs=None, stream=None):
+        """rosaq_linear_multi: the linears `weights` (same d_in / bits / k_salient) applied to one x in one launch."""
+        assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1
+        n = len(weights)
+        if outs is None:
+            outs = [torch.empty((x.shape[0], w.d_out), dtype=torch.float16, device=x.device) for w in weights]
+        wa = (C.c_void_p * n)(*[w._h.value for w in weights])
+        ya = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+        la = (C.c_int64 * n)(*[o.stride(0) for o in outs])
+        _check(lib().rosaq_linear_multi(self._h, _ptr(x), x.shape[0], x.stride(0),
+                                        None if rotation is None else rotation._h, n, wa, ya, la, _stream(stream)),
+               "rosaq_linear_multi")
+        return outs
+
     def linear_static(self, x, weight, rotation=None, out=None, stream=None):
         """rosaq_linear_static: same result as `linear`, but the library allocates nothing (the rotated
         activations live in a fixed 4 MiB array inside the library).  Pass `out`: with out=None this
@@ -300,6 +316,10 @@ def rosaq_rotate(ctx, x, rotation, out=None, stream=None):
 
 def rosaq_linear(ctx, x, weight, rotation=None, out=None, stream=None):
     return ctx.linear(x, weight, rotation, out, stream)
+
+
+def rosaq_linear_multi(ctx, x, weights, rotation=None, outs=None, stream=None):
+    return ctx.linear_multi(x, weights, rotation, outs, stream)
 
 
 def rosaq_linear_static(ctx, x, weight, rotation=None, out=None, stream=None):

@@ -34,17 +34,23 @@ constexpr int kFirstDequantWarp = 3;
 constexpr int kWSlotBytes = kInt4CodeBytes + kScaleBytes;  // 8704: one quantized tile or a quarter fp16 tile
 constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels of an fp16 tile
 constexpr int kTmemCols = 256;
+constexpr int kMaxProblems = 4;   // weights sharing one activation in a launch (q/k/v, gate/up)
 constexpr int kMaxSplits = 8;
 
 struct TcParams {
-  const uint8_t *blob;
+  // up to kMaxProblems weights of identical geometry (d_in, bits, salient groups) that multiply the same
+  // activations: their column tiles are laid side by side along gridDim.x
+  int n_prob;
+  int tile_start[kMaxProblems + 1];
+  const uint8_t *blob[kMaxProblems];
+  int d_out[kMaxProblems];
+  __half *y[kMaxProblems];
+  long long ldy[kMaxProblems];
   long long tile_stride;
-  int g_fp16, g_quant, bits, block_groups, d_out;
+  int g_fp16, g_quant, bits, block_groups;
   int M, MT;                 // tokens in the problem, tokens per CTA (multiple of 16, <= 128)
   int S;                     // K splits = cluster size along y
   int g_bounds[kMaxSplits + 1];
-  __half *y;
-  long long ldy;
   const int32_t *col_map;
   int *status;
   long long wait_limit;
@@ -163,21 +169,15 @@ __device__ __forceinline__ uint32_t cluster_rank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
-}
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(addr)
-               : "memory");
-  return v;
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -308,7 +308,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const uint32_t p_buf = base;                                 // fp32 partial tile, aliases the rings afterwards
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nt = blockIdx.x, split = blockIdx.y, m0 = blockIdx.z * MT;
+  int prob = 0;
+  while (prob + 1 < p.n_prob && (int)blockIdx.x >= p.tile_start[prob + 1]) ++prob;
+  const int nt = blockIdx.x - p.tile_start[prob], split = blockIdx.y, m0 = blockIdx.z * MT;
+  const int d_out = p.d_out[prob];
+  __half *const y_out = p.y[prob];
+  const long long ldy = p.ldy[prob];
   const int g_begin = p.g_bounds[split], g_end = p.g_bounds[split + 1];
   const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit};
 
@@ -338,7 +343,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const uint32_t tmem = misc_ptr[0];
   const uint32_t a_col0 = (MT <= 64) ? 64u : 128u;             // A buffers follow the accumulator columns
 
-  const uint8_t *tile_base = p.blob + (long long)nt * p.tile_stride;
+  const uint8_t *tile_base = p.blob[prob] + (long long)nt * p.tile_stride;
   const int qbytes = quant_tile_bytes(kBits);
 
   if (warp == 0) {
@@ -482,64 +487,99 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       tc_fence_before();
       mbar_arrive(bar_a_full + 8 * st);
     }
-    // ---------------- epilogue part 1: accumulators -> fp32 partial tile in shared memory
-    bool have_d = ok && ab.wait(bar_d_full, 0);
-    have_d = __all_sync(0xffffffffu, have_d);
+  }
+
+  // ---------------- epilogue
+  // Lane n of a dequantisation warp holds output column n of the tile; its TMEM columns are the tokens.
+  // S == 1: registers -> y.  S > 1: token row m of the tile is owned by cluster rank m % S; every CTA
+  // pushes the rows of its partial tile into the owners' shared memory (plain remote stores: no round
+  // trip), one cluster barrier later each owner adds the S contributions in rank order (so the sum
+  // does not depend on timing) and writes its rows of y.  The receive buffer reuses the operand rings,
+  // hence the first cluster barrier: every CTA of the cluster must be done with its main loop.
+  // All threads take the barriers whatever happened before; a CTA whose waits expired only skips the
+  // memory traffic.
+  const bool is_epi = warp >= kFirstDequantWarp;
+  const int quad = warp & 3, hf = is_epi ? (warp - kFirstDequantWarp) >> 2 : 0;
+  const int n = quad * 32 + lane;
+  const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+  const int half_cols = MT >> 1, col0 = hf * half_cols;
+  bool have_d = false;
+  if (is_epi) {
+    have_d = ab.wait(bar_d_full, 0);
+    have_d = __all_sync(0xffffffffu, have_d && !ab.set());
+    if (have_d) tc_fence_after();
+  }
+  if (p.S == 1) {
     if (have_d) {
-      tc_fence_after();
-      const int half_cols = MT >> 1;               // this warp's share of the token columns
+      grid_dep_wait();                                       // y may still be read by the previous kernel
+      const int n_glob = nt * kTileN + n;
+      const bool n_ok = n_glob < d_out;
+      const long long out_col = n_ok ? (p.col_map ? p.col_map[n_glob] : n_glob) : 0;
       for (int c0 = 0; c0 < half_cols; c0 += 8) {
         uint32_t v[8];
-        const int col = hf * half_cols + c0;
-        tmem_ld8(lane_addr + col, v);
+        tmem_ld8(lane_addr + col0 + c0, v);
         tc_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          *reinterpret_cast<uint32_t *>(gen + (p_buf - base) + ((col + e) * kTileN + n) * 4) = v[e];
+        for (int e = 0; e < 8; ++e) {
+          const int mg = m0 + col0 + c0 + e;
+          if (n_ok && mg < p.M) y_out[(long long)mg * ldy + out_col] = __float2half_rn(__uint_as_float(v[e]));
+        }
+      }
+    }
+  } else {
+    const uint32_t rank = cluster_rank();
+    const int rows_max = (MT + p.S - 1) / p.S;               // rows any rank can own
+    const uint32_t recv = base;                              // [source rank][row slot][128] fp32
+    cluster_arrive();                                        // #1: this CTA no longer touches its rings
+    cluster_wait();
+    if (have_d) {
+      // token m = col0 + c goes to rank m % S, row slot m / S; walked without division
+      int r = col0 % p.S, jrow = col0 / p.S;
+      for (int c0 = 0; c0 < half_cols; c0 += 8) {
+        uint32_t v[8];
+        tmem_ld8(lane_addr + col0 + c0, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t dst = recv + (uint32_t)(((int)rank * rows_max + jrow) * kTileN + n) * 4u;
+          st_cluster_u32(map_to_rank(dst, (uint32_t)r), v[e]);
+          if (++r == p.S) {
+            r = 0;
+            ++jrow;
+          }
+        }
+      }
+    }
+    cluster_arrive();                                        // #2: release my pushes, acquire everybody else's
+    cluster_wait();
+    if (is_epi && !ab.set()) {
+      grid_dep_wait();                                       // y may still be read by the previous kernel
+      const int tid = threadIdx.x - kFirstDequantWarp * 32;
+      const int rows = (MT - (int)rank + p.S - 1) / p.S;     // token rows rank, rank + S, ...
+      const int n0 = nt * kTileN;
+      for (int it = tid; it < rows * 32; it += kDequantThreads) {
+        const int jrow = it >> 5, i4 = it & 31;
+        const uint8_t *src = gen + (uint32_t)(jrow * kTileN + i4 * 4) * 4u;
+        float4 acc = *reinterpret_cast<const float4 *>(src);
+        for (int sp = 1; sp < p.S; ++sp) {
+          const float4 v = *reinterpret_cast<const float4 *>(src + (size_t)sp * rows_max * kTileN * 4);
+          acc.x += v.x, acc.y += v.y, acc.z += v.z, acc.w += v.w;
+        }
+        const int mg = m0 + (int)rank + jrow * p.S, nn = n0 + i4 * 4;
+        if (mg >= p.M || nn >= d_out) continue;
+        __align__(8) __half h[4] = {__float2half_rn(acc.x), __float2half_rn(acc.y), __float2half_rn(acc.z),
+                                    __float2half_rn(acc.w)};
+        __half *row = y_out + (long long)mg * ldy;
+        if (!p.col_map && nn + 3 < d_out) {
+          *reinterpret_cast<uint2 *>(row + nn) = *reinterpret_cast<const uint2 *>(h);
+        } else {
+          for (int e = 0; e < 4 && nn + e < d_out; ++e) row[p.col_map ? p.col_map[nn + e] : nn + e] = h[e];
+        }
       }
     }
   }
 
-  // ---------------- epilogue part 2: split-K sum over the cluster in rank order, fp16 store
   tc_fence_before();
-  __syncthreads();
-  if (p.S > 1) cluster_sync_all();
-  if (warp >= kFirstDequantWarp && !ab.set()) {
-    grid_dep_wait();                                         // y may still be read by the previous kernel
-    const int tid = threadIdx.x - kFirstDequantWarp * 32;
-    const uint32_t rank = p.S > 1 ? cluster_rank() : 0;
-    const int rows = (MT - (int)rank + p.S - 1) / p.S;    // token rows rank, rank+S, ...
-    const int n0 = nt * kTileN;
-    for (int it = tid; it < rows * 32; it += kDequantThreads) {
-      const int m = (int)rank + (it >> 5) * p.S, i4 = it & 31;
-      const uint32_t off = p_buf + (uint32_t)(m * kTileN + i4 * 4) * 4;
-      float4 acc;
-      if (p.S > 1) {
-        // all remote loads are issued before the first add (a DSMEM round trip each); the sum still
-        // runs in rank order
-        float4 v[kMaxSplits];
-#pragma unroll
-        for (int s = 0; s < kMaxSplits; ++s)
-          v[s] = s < p.S ? ld_cluster_f4(map_to_rank(off, s)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        acc = v[0];
-#pragma unroll
-        for (int s = 1; s < kMaxSplits; ++s)
-          if (s < p.S) acc.x += v[s].x, acc.y += v[s].y, acc.z += v[s].z, acc.w += v[s].w;
-      } else {
-        acc = *reinterpret_cast<const float4 *>(gen + (off - base));
-      }
-      const int mg = m0 + m, n = n0 + i4 * 4;
-      if (mg >= p.M || n >= p.d_out) continue;
-      __align__(8) __half h[4] = {__float2half_rn(acc.x), __float2half_rn(acc.y), __float2half_rn(acc.z), __float2half_rn(acc.w)};
-      __half *row = p.y + (long long)mg * p.ldy;
-      if (!p.col_map && n + 3 < p.d_out) {
-        *reinterpret_cast<uint2 *>(row + n) = *reinterpret_cast<const uint2 *>(h);
-      } else {
-        for (int e = 0; e < 4 && n + e < p.d_out; ++e) row[p.col_map ? p.col_map[n + e] : n + e] = h[e];
-      }
-    }
-  }
-  if (p.S > 1) cluster_sync_all();   // nobody leaves while a peer may still read its partial tile
   __syncthreads();
   if (warp == 2) {
     __syncwarp();
@@ -584,25 +624,48 @@ int tc_env_int(const char *name, int dflt) {
 
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
                      const int32_t *col_map, __half *y, long long ldy, cudaStream_t s) {
+  const TiledOperand *ts[1] = {&t};
+  __half *ys[1] = {y};
+  long long ldys[1] = {ldy};
+  return launch_linear_tc_multi(ctx, x, M, ldx, 1, ts, col_map, ys, ldys, s);
+}
+
+// n weights of identical geometry applied to the same activations in one launch
+int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, int n,
+                           const TiledOperand *const *ts, const int32_t *col_map, __half *const *ys,
+                           const long long *ldys, cudaStream_t s) {
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return ROSAQ_ERR_CUDA;
+  if (n < 1 || n > kMaxProblems) return ROSAQ_ERR_INVALID_ARG;
+  const TiledOperand &t = *ts[0];
   const int G = groups_per_tile(t);
   if (G <= 0) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
 
   TcParams p{};
-  p.blob = t.blob;
+  p.n_prob = n;
+  int n_tiles_all = 0;
+  for (int i = 0; i < n; ++i) {
+    const TiledOperand &ti = *ts[i];
+    if (ti.d_in != t.d_in || ti.g_fp16 != t.g_fp16 || ti.g_quant != t.g_quant || ti.block_groups != t.block_groups ||
+        (t.g_quant > 0 && ti.bits != t.bits))
+      return ROSAQ_ERR_INVALID_ARG;
+    p.tile_start[i] = n_tiles_all;
+    p.blob[i] = ti.blob;
+    p.d_out[i] = ti.d_out;
+    p.y[i] = ys[i];
+    p.ldy[i] = ldys[i];
+    n_tiles_all += ti.n_tiles;
+  }
+  p.tile_start[n] = n_tiles_all;
   p.tile_stride = t.tile_stride;
   p.g_fp16 = t.g_fp16;
   p.g_quant = t.g_quant;
   p.bits = t.bits;
   p.block_groups = t.block_groups;
-  p.d_out = t.d_out;
   p.M = M;
   const int m_tiles = (M + 127) / 128;
   const int per_tile = (M + m_tiles - 1) / m_tiles;
   p.MT = ((per_tile + 15) / 16) * 16;
-  p.y = y;
-  p.ldy = ldy;
   p.col_map = col_map;
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
@@ -617,7 +680,7 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
 
   // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
   // equal bytes (an fp16 group weighs four quantized ones)
-  const int tiles = t.n_tiles * m_tiles;
+  const int tiles = n_tiles_all * m_tiles;
   int S = (2 * ctx->sm_count) / (tiles > 0 ? tiles : 1);
   S = S < 1 ? 1 : (S > kMaxSplits ? kMaxSplits : S);
   if (S > G) S = G;
@@ -666,7 +729,7 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
     attr_smem[ki] = smem;
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(t.n_tiles, S, m_tiles);
+  cfg.gridDim = dim3(n_tiles_all, S, m_tiles);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;

@@ -375,4 +375,43 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
   return run_gemm(ctx, xin, M, ld, w->t, nullptr, static_cast<__half *>(y), ldy, s);
 }
 
+int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r, int n,
+                       const rosaq_weight *const *w, void *const *y, const int64_t *ldy, void *stream) {
+  if (!ctx || !w || !y || !ldy || n < 1 || n > 4) return ROSAQ_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (!w[i]) return ROSAQ_ERR_INVALID_ARG;
+  int st = check_act(x, M, ldx, w[0]->t.d_in);
+  for (int i = 0; i < n && st == ROSAQ_OK; ++i) {
+    const TiledOperand &a = w[i]->t, &b = w[0]->t;
+    if (a.d_in != b.d_in || a.g_fp16 != b.g_fp16 || a.g_quant != b.g_quant || (b.g_quant > 0 && a.bits != b.bits))
+      return ROSAQ_ERR_INVALID_ARG;
+    st = check_act(y[i], M, ldy[i], a.d_out);
+  }
+  if (st != ROSAQ_OK) return st;
+  if (r && r->d != w[0]->t.d_in) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __half *xin = static_cast<const __half *>(x);
+  long long ld = ldx;
+  if (r) {
+    st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
+    if (st != ROSAQ_OK) return st;
+    st = run_gemm(ctx, xin, M, ldx, r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d, s);
+    if (st != ROSAQ_OK) return st;
+    xin = static_cast<const __half *>(ctx->ws);
+    ld = r->d;
+  }
+  if (ctx->impl == 1) {
+    for (int i = 0; i < n && st == ROSAQ_OK; ++i)
+      st = launch_linear_simt(ctx, xin, M, ld, w[i]->t, nullptr, static_cast<__half *>(y[i]), ldy[i], s);
+    return st;
+  }
+  const TiledOperand *ts[4];
+  __half *ys[4];
+  long long ldys[4];
+  for (int i = 0; i < n; ++i) ts[i] = &w[i]->t, ys[i] = static_cast<__half *>(y[i]), ldys[i] = ldy[i];
+  return launch_linear_tc_multi(ctx, xin, M, ld, n, ts, nullptr, ys, ldys, s);
+}
+
 }  // extern "C"

@@ -220,5 +220,8 @@ int launch_linear_simt(const rosaq_ctx *ctx, const __half *x, int M, long long l
                        const int32_t *col_map, __half *y, long long ldy, cudaStream_t s);
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
                      const int32_t *col_map, __half *y, long long ldy, cudaStream_t s);
+int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, int n,
+                           const TiledOperand *const *ts, const int32_t *col_map, __half *const *ys,
+                           const long long *ldys, cudaStream_t s);
 
 }  // namespace rosaq

@@ -142,6 +142,29 @@ def test_linear_strided_activations_and_output(ctx):
     assert torch.all(ybuf[:, 512:] == 7.0)       # nothing written past d_out
 
 
+@pytest.mark.parametrize("bits,M", [(4, 64), (3, 5), (4, 200)])
+def test_linear_multi_gives_the_bits_of_separate_calls(ctx, bits, M):
+    """q/k/v-style: three weights of different widths on one activation, one launch, with and without R."""
+    c = H.config_tiny()
+    widths = [512, 200, 136]
+    Ws = [synth.weights(512, n, seed=51, key=f"multi{n}", outlier_frac=0.01) for n in widths]
+    ws = [ctx.quantize(dev(W), dev(c["R32"]), bits=bits, k_salient=128) for W in Ws]
+    rot = ctx.rotation_create(dev(c["R16"]))
+    x = dev(synth.ActivationLaw(512, 1.2, 0, "tiny", mix="qr").sample(M, "xm", np.float16))
+    want = [ctx.linear(x, w, rot).cpu().numpy() for w in ws]
+    got = ctx.linear_multi(x, ws, rot)
+    xr = ctx.rotate(x, rot)
+    got2 = ctx.linear_multi(xr, ws, None)
+    check_status(ctx)
+    for a, b, b2 in zip(want, got, got2):
+        assert np.array_equal(a.view(np.uint16), b.cpu().numpy().view(np.uint16))
+        assert np.array_equal(a.view(np.uint16), b2.cpu().numpy().view(np.uint16))
+    with pytest.raises(rb.RosaqError) as e:                  # mismatched geometry is an error code
+        other = ctx.quantize(dev(Ws[0]), dev(c["R32"]), bits=bits, k_salient=256)
+        ctx.linear_multi(x, [ws[0], other], rot)
+    assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+
+
 def test_special_case_all_salient_is_plain_fp16_gemm(ctx):
     rng = np.random.default_rng(12)
     W = (rng.standard_normal((256, 128)) * 0.02).astype(np.float16)
