@@ -239,21 +239,24 @@ def profile_shape(args):
     d_in, d_out, M, bits = args.profile_shape
     ctx = rb.Context(0)
     g = torch.Generator(device="cuda").manual_seed(0)
-    nq = d_in - K_SALIENT
-    nw = nq // 8 if bits == 4 else nq // 32 * 3
+    ks = d_in if bits == 16 else K_SALIENT            # bits 16: every group fp16 (the shape of a rotation operand)
+    qbits = 4 if bits == 16 else bits
+    nq = d_in - ks
+    nw = nq // 8 if qbits == 4 else nq // 32 * 3
     qw = torch.randint(-2 ** 31, 2 ** 31 - 1, (nw, d_out), dtype=torch.int64, device="cuda", generator=g).to(torch.int32)
     sc = (torch.rand((nq // 128, d_out), device="cuda", generator=g) * 0.01 + 0.001).half()
-    zr = torch.randint(0, 2 ** bits, (nq // 128, d_out), device="cuda", generator=g).half()
-    sal = (torch.randn((K_SALIENT, d_out), device="cuda", generator=g) * 0.02).half()
-    w0 = ctx.weight_import(d_in, d_out, bits, 128, K_SALIENT, qw, sc, zr, sal)
+    zr = torch.randint(0, 2 ** qbits, (nq // 128, d_out), device="cuda", generator=g).half()
+    sal = (torch.randn((ks, d_out), device="cuda", generator=g) * 0.02).half()
+    mk = lambda: ctx.weight_import(d_in, d_out, qbits, 128, ks, qw, sc, zr, sal)
+    w0 = mk()
     copies = args.copies or max(2, int(np.ceil(2 * 126e6 / w0.device_bytes)))
-    ws = [w0] + [ctx.weight_import(d_in, d_out, bits, 128, K_SALIENT, qw, sc, zr, sal) for _ in range(copies - 1)]
+    ws = [w0] + [mk() for _ in range(copies - 1)]
     x = torch.randn((M, d_in), device="cuda", generator=g).half()
     y = torch.empty((M, d_out), dtype=torch.float16, device="cuda")
     gph = capture(lambda: [ctx.linear(x, w, None, out=y) for w in ws])
     ts = sorted(time_graphs([gph], 1, 1) * 1e3 / copies for _ in range(args.steps))
     us = ts[len(ts) // 2]
-    nb = gemm_bytes(d_in, d_out, M, bits)
+    nb = gemm_bytes(d_in, d_out, M, qbits, ks)
     assert ctx.last_status() == 0
     print(json.dumps({"shape": f"{d_in}x{d_out}", "M": M, "bits": bits, "copies": copies, "us": round(us, 3),
                       "us_min": round(ts[0], 3), "gbs": round(nb / us / 1e3, 1),
