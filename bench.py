@@ -263,6 +263,33 @@ def profile_shape(args):
                       "tflops": round(2.0 * M * d_in * d_out / us / 1e6, 1)}))
 
 
+def calib_cov_throughput(ctx, peaks, n_tokens=16384, d=5120, reps=5):
+    """rosaq_calib_cov on one chunk of the 13B-shaped calibration stream (fp16 activations, fp32 C):
+    device time per call and tensor throughput.  `tflops` counts the multiply-adds the kernel executes
+    (the 128 x 128 tiles of the lower triangle, diagonal included); `tflops_full_square` credits the
+    whole d x d result that those tiles produce by symmetry."""
+    import torch
+    X = torch.randn((n_tokens, d), device="cuda", dtype=torch.float16)
+    Cm = torch.zeros((d, d), dtype=torch.float32, device="cuda")
+    ctx.calib_cov(X, Cm)
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.calib_cov(X, Cm)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    ms = sorted(ts)[len(ts) // 2]
+    nt = (d + 127) // 128
+    executed = 2.0 * n_tokens * 128 * 128 * (nt * (nt + 1) // 2)
+    tf = executed / ms / 1e9
+    return dict(tokens=n_tokens, d=d, ms=round(ms, 4), tflops=round(tf, 1),
+                tflops_full_square=round(2.0 * n_tokens * d * d / ms / 1e9, 1),
+                frac_of_bf16_peak=round(tf / peaks["bf16_tflops"], 4), peak_source=peaks["source"])
+
+
 # ----------------------------------------------------------------------------- oracle legs
 def oracle_sample(bits, seconds_hint=15.0):
     """Times the CPU oracle's forward (fp64, dequantise on the fly) on a column sample of the
@@ -388,6 +415,7 @@ def run_ours(args):
     }
     if not args.no_table:
         line["gemm_stage"] = gemm_stage_table(ctx, model, args.bits, peaks)
+        line["calib_cov"] = calib_cov_throughput(ctx, peaks)
     if not args.no_cpu_baseline and world == 1:
         v, cores, text = oracle_sample(args.bits)
         line["cpu_baseline"] = {"value": round(v, 4), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": text}
@@ -405,12 +433,18 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-shape", type=int, nargs=4, metavar=("D_IN", "D_OUT", "M", "BITS"),
                     help="time the GEMM stage alone on one shape (random weights) and exit")
+    ap.add_argument("--profile-cov", type=int, nargs=2, metavar=("TOKENS", "D"),
+                    help="time rosaq_calib_cov alone on TOKENS x D fp16 activations and exit")
     ap.add_argument("--copies", type=int, default=0, help="--profile-shape: distinct weight copies (default: 2 x L2)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.profile_shape:
         args.steps = min(args.steps, 30)
         return profile_shape(args)
+    if args.profile_cov:
+        from paper_2506_13472_b200 import binding as rb
+        print(json.dumps(calib_cov_throughput(rb.Context(0), load_peaks(), *args.profile_cov)))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

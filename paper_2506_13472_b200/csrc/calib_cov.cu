@@ -1,11 +1,312 @@
 // Eq. 4, left-hand side: the calibration Gram matrix C += X^T X.
+//
+// fp16 activations go to the tensor cores (tcgen05): the Gram matrix is a symmetric rank-N update,
+// C[i][j] = sum_t X[t][i] X[t][j], so both MMA operands are slices of the same row-major X with
+// the token index as the contraction dimension -- "MN-major" operands, which TMA delivers directly
+// (box = 64 channels x 64 tokens, 128-byte swizzle) without any transposition.  One CTA owns one
+// 128 x 128 tile of the lower triangle of one head block and walks over all tokens of the call with
+// fp32 accumulators in tensor memory; diagonal tiles load one operand and use it twice.  The
+// epilogue adds the tile to C and, for off-diagonal tiles, its transpose to the mirrored position,
+// so both triangles are written and C stays exactly symmetric.
+//
+// fp32 activations (and blocks narrower than 64 channels) keep the CUDA-core path of quantize.cu,
+// whose products are exact.
+//
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue.
+// Every wait is bounded (ROSAQ_ERR_TIMEOUT through the context's status word).
+#include <cuda.h>
+
 #include "rosaq_internal.cuh"
 
 namespace rosaq {
 
-int launch_cov(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
-               cudaStream_t s) {
-  return launch_cov_fma(X, x_dtype, n_tokens, d, ldx, n_blocks, C, s);
+namespace {
+
+constexpr int kCovTile = 128;      // output tile edge
+constexpr int kCovTokens = 64;     // tokens per pipeline stage
+constexpr int kCovStages = 4;
+constexpr int kCovThreads = 192;
+constexpr int kBoxBytes = 64 * kCovTokens * 2;          // one TMA box: 64 channels x 64 tokens fp16
+constexpr int kOperandBytes = 2 * kBoxBytes;            // 128 channels
+constexpr int kStageBytes = 2 * kOperandBytes;          // A and B
+constexpr uint32_t kCovTmemCols = 128;
+
+struct CovParams {
+  float *C;
+  int dh, n_tile;              // block edge, tiles per block edge
+  long long n_tokens;
+  int *status;
+  long long wait_limit;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(1000u)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
+          "r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// MN-major operand, 128-byte swizzle: 64-channel blocks kBoxBytes apart (leading offset), groups of
+// 8 tokens 1024 bytes apart (stride offset).
+__device__ __forceinline__ uint64_t make_mn_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3fff) | ((uint64_t)(kBoxBytes >> 4) << 16) | (64ull << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+
+// four MMAs = one stage of 64 tokens; descriptors advance by 16 tokens = 2048 bytes = 128 units of 16 bytes
+__device__ __forceinline__ void tc_mma4_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 ta, tb;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "add.u64 ta, %1, 128;\n\tadd.u64 tb, %2, 128;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], ta, tb, %3, q;\n\t"
+      "add.u64 ta, %1, 256;\n\tadd.u64 tb, %2, 256;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], ta, tb, %3, q;\n\t"
+      "add.u64 ta, %1, 384;\n\tadd.u64 tb, %2, 384;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], ta, tb, %3, q;\n\t}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+struct CovAbort {
+  volatile int *flag;
+  int *status;
+  long long limit;
+  __device__ __forceinline__ bool set() const { return *flag != 0; }
+  __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (long long it = 0; it < limit; ++it) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((it & 63) == 63 && set()) return false;
+    }
+    *flag = 1;
+    atomicExch(status, (int)ROSAQ_ERR_TIMEOUT);
+    return false;
+  }
+};
+
+__global__ void __launch_bounds__(kCovThreads, 1)
+cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ uint64_t bars[2 * kCovStages + 1];
+  __shared__ uint32_t misc[2];                       // [0] TMEM base, [1] abort flag
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[kCovStages]);
+  const uint32_t bar_d = smem_u32(&bars[2 * kCovStages]);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const CovAbort ab{reinterpret_cast<volatile int *>(&misc[1]), p.status, p.wait_limit};
+
+  // tile (bi >= bj) of the lower triangle from the linear index: bi(bi+1)/2 + bj
+  int bi = 0;
+  {
+    const int t = blockIdx.x;
+    while ((bi + 1) * (bi + 2) / 2 <= t) ++bi;
+  }
+  const int bj = blockIdx.x - bi * (bi + 1) / 2;
+  const int h = blockIdx.y;
+  const bool diag = bi == bj;
+  const int col_a = h * p.dh + bi * kCovTile, col_b = h * p.dh + bj * kCovTile;
+  const int n_stages_total = (int)((p.n_tokens + kCovTokens - 1) / kCovTokens);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kCovStages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    mbar_init(bar_d, 1);
+    misc[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc[0])),
+                 "n"(kCovTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = 0, idx = 0;
+      uint32_t lap = 0;
+      for (int s = 0; s < n_stages_total && !ab.set(); ++s, ++issued) {
+        if (!ab.wait(bar_empty + 8 * idx, lap ^ 1u)) break;
+        const uint32_t dst = base + idx * kStageBytes;
+        const int tok = s * kCovTokens;
+        mbar_arrive_expect_tx(bar_full + 8 * idx, diag ? kOperandBytes : kStageBytes);
+        tma_load_2d(dst, &xmap, bar_full + 8 * idx, col_a, tok);
+        tma_load_2d(dst + kBoxBytes, &xmap, bar_full + 8 * idx, col_a + 64, tok);
+        if (!diag) {
+          tma_load_2d(dst + kOperandBytes, &xmap, bar_full + 8 * idx, col_b, tok);
+          tma_load_2d(dst + kOperandBytes + kBoxBytes, &xmap, bar_full + 8 * idx, col_b + 64, tok);
+        }
+        if (++idx == kCovStages) idx = 0, lap ^= 1u;
+      }
+      if (ab.set()) {  // let loads already in flight land before the CTA goes away
+        for (int back = 1; back <= kCovStages && back <= issued; ++back) {
+          const int u = issued - back;
+          for (long long it = 0; it < p.wait_limit; ++it)
+            if (mbar_try_wait(bar_full + 8 * (u % kCovStages), (u / kCovStages) & 1)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // fp16 x fp16 -> fp32, both operands MN-major, M = N = 128
+      const uint32_t idesc = (1u << 4) | (1u << 15) | (1u << 16) | ((uint32_t)(kCovTile >> 3) << 17) |
+                             ((uint32_t)(kCovTile >> 4) << 24);
+      int idx = 0;
+      uint32_t lap = 0, accumulate = 0;
+      for (int s = 0; s < n_stages_total; ++s) {
+        if (!ab.wait(bar_full + 8 * idx, lap)) break;
+        tc_fence_after();
+        const uint32_t a_addr = base + idx * kStageBytes;
+        const uint64_t a = make_mn_desc(a_addr), b = diag ? a : make_mn_desc(a_addr + kOperandBytes);
+        tc_mma4_ss(tmem, a, b, idesc, accumulate);
+        accumulate = 1;
+        tc_commit(bar_empty + 8 * idx);
+        if (++idx == kCovStages) idx = 0, lap ^= 1u;
+      }
+      tc_commit(bar_d);
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> shared (transposable staging) -> C += tile, C^T += tile^T
+    const int quad = warp & 3;                        // warps 2..5 cover the four lane quadrants
+    const int row = quad * 32 + lane;                 // tile row i = TMEM lane
+    bool have = ab.wait(bar_d, 0);
+    have = __all_sync(0xffffffffu, have && !ab.set());
+    float *stage = reinterpret_cast<float *>(gen);    // [128][129] fp32, reuses the operand ring
+    constexpr int kPitch = kCovTile + 1;
+    if (have) {
+      tc_fence_after();
+      const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+      for (int c0 = 0; c0 < kCovTile; c0 += 8) {
+        uint32_t v[8];
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "r"(lane_addr + c0)
+                     : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int e = 0; e < 8; ++e) stage[row * kPitch + c0 + e] = __uint_as_float(v[e]);
+      }
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");    // the four epilogue warps
+    if (!ab.set()) {
+      const int tid = threadIdx.x - 64;               // 0..127
+      float *Cb = p.C + (long long)h * p.dh * p.dh;
+      const int i0 = bi * kCovTile, j0 = bj * kCovTile;
+      // C[i0 + r][j0 + tid] += tile[r][tid]: a warp touches 32 consecutive floats of one row of C
+      if (j0 + tid < p.dh) {
+        for (int r = 0; r < kCovTile && i0 + r < p.dh; ++r) {
+          float *c = Cb + (long long)(i0 + r) * p.dh + j0 + tid;
+          *c = __fadd_rn(*c, stage[r * kPitch + tid]);
+        }
+      }
+      // mirror: C[j0 + r][i0 + tid] += tile[tid][r]
+      if (!diag && i0 + tid < p.dh) {
+        for (int r = 0; r < kCovTile && j0 + r < p.dh; ++r) {
+          float *c = Cb + (long long)(j0 + r) * p.dh + i0 + tid;
+          *c = __fadd_rn(*c, stage[tid * kPitch + r]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kCovTmemCols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn cov_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+    else
+      (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+}  // namespace
+
+int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks,
+               float *C, cudaStream_t s) {
+  const int dh = d / n_blocks;
+  EncodeTiledFn encode = cov_encode_fn();
+  if (x_dtype != ROSAQ_F16 || dh < 64 || !encode || n_tokens > 0x7fffffffll)
+    return launch_cov_fma(X, x_dtype, n_tokens, d, ldx, n_blocks, C, s);
+
+  CUtensorMap xmap;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n_tokens};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kCovTokens};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(X), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
+  }
+  CovParams p{};
+  p.C = C;
+  p.dh = dh;
+  p.n_tile = (dh + kCovTile - 1) / kCovTile;
+  p.n_tokens = n_tokens;
+  p.status = ctx->d_status;
+  p.wait_limit = ctx->wait_limit;
+  const size_t smem = 1024 + (size_t)kCovStages * kStageBytes;   // the 128 x 129 fp32 staging tile fits inside
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return ROSAQ_ERR_CUDA;
+    }
+    attr_done = true;
+  }
+  dim3 grid(p.n_tile * (p.n_tile + 1) / 2, n_blocks);
+  cov_tc_kernel<<<grid, kCovThreads, smem, s>>>(xmap, p);
+  return cudaGetLastError() == cudaSuccess ? ROSAQ_OK : ROSAQ_ERR_CUDA;
 }
 
 }  // namespace rosaq

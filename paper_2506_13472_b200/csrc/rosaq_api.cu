@@ -174,7 +174,7 @@ int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens
   if (n_tokens == 0) return ROSAQ_OK;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return ROSAQ_ERR_CUDA;
-  return launch_cov(X, x_dtype, n_tokens, d, ldx, n_blocks, C, static_cast<cudaStream_t>(stream));
+  return launch_cov(ctx, X, x_dtype, n_tokens, d, ldx, n_blocks, C, static_cast<cudaStream_t>(stream));
 }
 
 int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, int bits,

@@ -214,8 +214,8 @@ int launch_rotation_tiles(const __half *q, int d, int n_blocks, const TiledOpera
 int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, cudaStream_t s);
 int launch_cov_fma(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
                    cudaStream_t s);
-int launch_cov(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
-               cudaStream_t s);
+int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tokens, int d, long long ldx,
+               int n_blocks, float *C, cudaStream_t s);
 int launch_linear_simt(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
                        const int32_t *col_map, __half *y, long long ldy, cudaStream_t s);
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
