@@ -307,7 +307,7 @@ def oracle_sample(bits, seconds_hint=15.0):
         orc.forward(x, qd)
         reps += 1
         dt = time.perf_counter() - t0
-        if dt > seconds_hint or reps >= 50:
+        if dt > seconds_hint or reps >= 5000:
             break
     nb = gemm_bytes(d, n_cols, M_TOKENS, bits) * reps
     return nb / dt / 1e9, orc.num_threads(), (f"oracle forward (fp64) on {n_cols} of 4096 output columns of the "
@@ -425,8 +425,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--bits", type=int, default=4, choices=[3, 4])
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape GEMM-stage / cuBLAS table")

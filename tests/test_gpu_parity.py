@@ -176,14 +176,7 @@ def test_special_case_all_salient_is_plain_fp16_gemm(ctx):
 
 
 # --------------------------------------------------------------------------- calib_cov
-def cov_tolerance(Cref, n_tokens):
-    """Products are exact in fp32 (fp16 x fp16) or rounded once (fp32 inputs); what is left is the fp32
-    accumulation.  CUDA-core path: N sequential roundings, ~sqrt(N) u in practice.  Tensor-core path:
-    one accumulator update per 16 tokens, each within one unit in the last place (2^-23) of the running
-    sum, which Cauchy-Schwarz bounds by sqrt(C_ii C_jj).  The bound below covers both."""
-    dg = np.sqrt(np.clip(np.diagonal(Cref, axis1=-2, axis2=-1), 0, None))
-    steps = max(4.0 * np.sqrt(n_tokens) + 8.0, 2.0 * (n_tokens / 16.0 + 8.0))
-    return 2.0 ** -24 * steps * dg[..., :, None] * dg[..., None, :]
+cov_tolerance = H.cov_tolerance
 
 
 @pytest.mark.parametrize("dtype,n_tokens,d,n_blocks", [
