@@ -4,10 +4,13 @@
 // C[i][j] = sum_t X[t][i] X[t][j], so both MMA operands are slices of the same row-major X with
 // the token index as the contraction dimension -- "MN-major" operands, which TMA delivers directly
 // (box = 64 channels x 64 tokens, 128-byte swizzle) without any transposition.  One CTA owns one
-// 128 x 128 tile of the lower triangle of one head block and walks over all tokens of the call with
-// fp32 accumulators in tensor memory; diagonal tiles load one operand and use it twice.  The
-// epilogue adds the tile to C and, for off-diagonal tiles, its transpose to the mirrored position,
-// so both triangles are written and C stays exactly symmetric.
+// 128 x 256 tile (128 x 128 for blocks of at most 128 channels) of one head block and walks over all
+// tokens of the call with fp32 accumulators in tensor memory.  Only tiles that touch the lower
+// triangle are computed: with 128-row blocks bi and 256-column blocks bj those are bj <= bi / 2.
+// A tile with bj == bi / 2 sits on the diagonal: its rows are a slice of its own columns, so it loads
+// one operand and uses it twice, and every element of its 256 x 256 diagonal block is produced
+// directly by it or its sibling.  The other tiles add themselves to C and their transpose to the
+// mirrored position.  Both triangles are therefore written and C stays exactly symmetric.
 //
 // fp32 activations (and blocks narrower than 64 channels) keep the CUDA-core path of quantize.cu,
 // whose products are exact.
@@ -22,18 +25,18 @@ namespace rosaq {
 
 namespace {
 
-constexpr int kCovTile = 128;      // output tile edge
+constexpr int kCovTile = 128;      // output tile rows (MMA M)
 constexpr int kCovTokens = 64;     // tokens per pipeline stage
 constexpr int kCovStages = 4;
 constexpr int kCovThreads = 192;
 constexpr int kBoxBytes = 64 * kCovTokens * 2;          // one TMA box: 64 channels x 64 tokens fp16
-constexpr int kOperandBytes = 2 * kBoxBytes;            // 128 channels
-constexpr int kStageBytes = 2 * kOperandBytes;          // A and B
-constexpr uint32_t kCovTmemCols = 128;
+constexpr int kOperandBytes = 2 * kBoxBytes;            // 128 channels (operand A)
+constexpr int kStageBytes = 6 * kBoxBytes;              // A (2 boxes) and up to 256 channels of B (4 boxes)
+constexpr uint32_t kCovTmemCols = 256;
 
 struct CovParams {
   float *C;
-  int dh, n_tile;              // block edge, tiles per block edge
+  int dh, bn;                  // block edge; tile columns (MMA N): 256, or 128 for narrow blocks
   long long n_tokens;
   int *status;
   long long wait_limit;
@@ -119,16 +122,20 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const CovAbort ab{reinterpret_cast<volatile int *>(&misc[1]), p.status, p.wait_limit};
 
-  // tile (bi >= bj) of the lower triangle from the linear index: bi(bi+1)/2 + bj
-  int bi = 0;
-  {
-    const int t = blockIdx.x;
-    while ((bi + 1) * (bi + 2) / 2 <= t) ++bi;
+  // row block bi (128 channels) has the column blocks bj = 0 .. bi / ratio (ratio = bn / 128)
+  const int ratio = p.bn / kCovTile;
+  int bi = 0, first = 0;
+  while (first + bi / ratio + 1 <= (int)blockIdx.x) {
+    first += bi / ratio + 1;
+    ++bi;
   }
-  const int bj = blockIdx.x - bi * (bi + 1) / 2;
+  const int bj = blockIdx.x - first;
   const int h = blockIdx.y;
-  const bool diag = bi == bj;
-  const int col_a = h * p.dh + bi * kCovTile, col_b = h * p.dh + bj * kCovTile;
+  const bool diag = bj == bi / ratio;
+  const int col_a = h * p.dh + bi * kCovTile, col_b = h * p.dh + bj * p.bn;
+  const int b_boxes = p.bn / 64;
+  // on a diagonal tile operand A is the slice of B that holds row block bi
+  const uint32_t a_in_b = diag ? (uint32_t)((bi % ratio) * kOperandBytes) : 0u;
   const int n_stages_total = (int)((p.n_tokens + kCovTokens - 1) / kCovTokens);
 
   if (threadIdx.x == 0) {
@@ -160,13 +167,13 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
         if (!ab.wait(bar_empty + 8 * idx, lap ^ 1u)) break;
         const uint32_t dst = base + idx * kStageBytes;
         const int tok = s * kCovTokens;
-        mbar_arrive_expect_tx(bar_full + 8 * idx, diag ? kOperandBytes : kStageBytes);
-        tma_load_2d(dst, &xmap, bar_full + 8 * idx, col_a, tok);
-        tma_load_2d(dst + kBoxBytes, &xmap, bar_full + 8 * idx, col_a + 64, tok);
+        mbar_arrive_expect_tx(bar_full + 8 * idx, (uint32_t)((diag ? 0 : 2) + b_boxes) * kBoxBytes);
         if (!diag) {
-          tma_load_2d(dst + kOperandBytes, &xmap, bar_full + 8 * idx, col_b, tok);
-          tma_load_2d(dst + kOperandBytes + kBoxBytes, &xmap, bar_full + 8 * idx, col_b + 64, tok);
+          tma_load_2d(dst, &xmap, bar_full + 8 * idx, col_a, tok);
+          tma_load_2d(dst + kBoxBytes, &xmap, bar_full + 8 * idx, col_a + 64, tok);
         }
+        for (int b = 0; b < b_boxes; ++b)
+          tma_load_2d(dst + kOperandBytes + b * kBoxBytes, &xmap, bar_full + 8 * idx, col_b + 64 * b, tok);
         if (++idx == kCovStages) idx = 0, lap ^= 1u;
       }
       if (ab.set()) {  // let loads already in flight land before the CTA goes away
@@ -179,16 +186,17 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // fp16 x fp16 -> fp32, both operands MN-major, M = N = 128
-      const uint32_t idesc = (1u << 4) | (1u << 15) | (1u << 16) | ((uint32_t)(kCovTile >> 3) << 17) |
+      // fp16 x fp16 -> fp32, both operands MN-major, M = 128, N = bn
+      const uint32_t idesc = (1u << 4) | (1u << 15) | (1u << 16) | ((uint32_t)(p.bn >> 3) << 17) |
                              ((uint32_t)(kCovTile >> 4) << 24);
       int idx = 0;
       uint32_t lap = 0, accumulate = 0;
       for (int s = 0; s < n_stages_total; ++s) {
         if (!ab.wait(bar_full + 8 * idx, lap)) break;
         tc_fence_after();
-        const uint32_t a_addr = base + idx * kStageBytes;
-        const uint64_t a = make_mn_desc(a_addr), b = diag ? a : make_mn_desc(a_addr + kOperandBytes);
+        const uint32_t b_addr = base + idx * kStageBytes + kOperandBytes;
+        const uint64_t b = make_mn_desc(b_addr);
+        const uint64_t a = make_mn_desc(diag ? b_addr + a_in_b : b_addr - kOperandBytes);
         tc_mma4_ss(tmem, a, b, idesc, accumulate);
         accumulate = 1;
         tc_commit(bar_empty + 8 * idx);
@@ -202,12 +210,12 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
     const int row = quad * 32 + lane;                 // tile row i = TMEM lane
     bool have = ab.wait(bar_d, 0);
     have = __all_sync(0xffffffffu, have && !ab.set());
-    float *stage = reinterpret_cast<float *>(gen);    // [128][129] fp32, reuses the operand ring
-    constexpr int kPitch = kCovTile + 1;
+    float *stage = reinterpret_cast<float *>(gen);    // [128][bn + 1] fp32, reuses the operand ring
+    const int pitch = p.bn + 1;
     if (have) {
       tc_fence_after();
       const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-      for (int c0 = 0; c0 < kCovTile; c0 += 8) {
+      for (int c0 = 0; c0 < p.bn; c0 += 8) {
         uint32_t v[8];
         asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
@@ -215,26 +223,38 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
                      : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int e = 0; e < 8; ++e) stage[row * kPitch + c0 + e] = __uint_as_float(v[e]);
+        for (int e = 0; e < 8; ++e) stage[row * pitch + c0 + e] = __uint_as_float(v[e]);
       }
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");    // the four epilogue warps
     if (!ab.set()) {
       const int tid = threadIdx.x - 64;               // 0..127
       float *Cb = p.C + (long long)h * p.dh * p.dh;
-      const int i0 = bi * kCovTile, j0 = bj * kCovTile;
-      // C[i0 + r][j0 + tid] += tile[r][tid]: a warp touches 32 consecutive floats of one row of C
-      if (j0 + tid < p.dh) {
-        for (int r = 0; r < kCovTile && i0 + r < p.dh; ++r) {
-          float *c = Cb + (long long)(i0 + r) * p.dh + j0 + tid;
-          *c = __fadd_rn(*c, stage[r * kPitch + tid]);
+      const int i0 = bi * kCovTile, j0 = bj * p.bn;
+      // C[i0 + r][j0 + c] += tile[r][c]: a warp touches 32 consecutive floats of one row of C
+      // (eight independent loads in flight per thread before the adds: the update is latency-bound)
+      const int n_rows = min(kCovTile, p.dh - i0), n_cols = min(p.bn, p.dh - j0);
+      for (int c = tid; c < n_cols; c += 128) {
+        float *dst = Cb + (long long)i0 * p.dh + j0 + c;
+        for (int r0 = 0; r0 < n_rows; r0 += 8) {
+          float old[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) old[e] = r0 + e < n_rows ? __ldcg(dst + (long long)(r0 + e) * p.dh) : 0.0f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (r0 + e < n_rows) dst[(long long)(r0 + e) * p.dh] = __fadd_rn(old[e], stage[(r0 + e) * pitch + c]);
         }
       }
-      // mirror: C[j0 + r][i0 + tid] += tile[tid][r]
-      if (!diag && i0 + tid < p.dh) {
-        for (int r = 0; r < kCovTile && j0 + r < p.dh; ++r) {
-          float *c = Cb + (long long)(j0 + r) * p.dh + i0 + tid;
-          *c = __fadd_rn(*c, stage[tid * kPitch + r]);
+      // mirror: C[j0 + c][i0 + tid] += tile[tid][c]
+      if (!diag && tid < n_rows) {
+        float *dst = Cb + (long long)j0 * p.dh + i0 + tid;
+        for (int c0 = 0; c0 < n_cols; c0 += 8) {
+          float old[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) old[e] = c0 + e < n_cols ? __ldcg(dst + (long long)(c0 + e) * p.dh) : 0.0f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (c0 + e < n_cols) dst[(long long)(c0 + e) * p.dh] = __fadd_rn(old[e], stage[tid * pitch + c0 + e]);
         }
       }
     }
@@ -291,11 +311,11 @@ int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tok
   CovParams p{};
   p.C = C;
   p.dh = dh;
-  p.n_tile = (dh + kCovTile - 1) / kCovTile;
+  p.bn = dh > kCovTile ? 256 : 128;
   p.n_tokens = n_tokens;
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
-  const size_t smem = 1024 + (size_t)kCovStages * kStageBytes;   // the 128 x 129 fp32 staging tile fits inside
+  const size_t smem = 1024 + (size_t)kCovStages * kStageBytes;   // the 128 x (bn + 1) fp32 staging tile fits inside
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -304,7 +324,10 @@ int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tok
     }
     attr_done = true;
   }
-  dim3 grid(p.n_tile * (p.n_tile + 1) / 2, n_blocks);
+  const int n_row_blocks = (dh + kCovTile - 1) / kCovTile, ratio = p.bn / kCovTile;
+  int tiles = 0;
+  for (int bi = 0; bi < n_row_blocks; ++bi) tiles += bi / ratio + 1;
+  dim3 grid(tiles, n_blocks);
   cov_tc_kernel<<<grid, kCovThreads, smem, s>>>(xmap, p);
   return cudaGetLastError() == cudaSuccess ? ROSAQ_OK : ROSAQ_ERR_CUDA;
 }
