@@ -35,6 +35,9 @@ UNIT = "GB/s"
 M_TOKENS = 64
 K_SALIENT = 128
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 7 launches of an INT4 step
+# (ncu capture of this command, summarised in profiles/bench_launch_list_7b_layer_m64.md)
+TRAFFIC_BYTES_PER_LAUNCH = 31578441
 
 
 # ----------------------------------------------------------------------------- bytes / flops
@@ -409,7 +412,8 @@ def run_ours(args):
         "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": round(e2e_ms, 5)},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                     "frac": round(achieved / peaks["hbm_gbs"], 4),
+                     "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.bits == 4 else None,
                      "peak_source": peaks["source"], "kernel": "linear_tc_kernel<4> (all 7 launches of a step: 3 rotations, qkv, o, gate+up, down)",
                      "frac_of_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)},
     }
