@@ -684,7 +684,9 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
   // equal bytes (an fp16 group weighs four quantized ones)
   const int tiles = n_tiles_all * m_tiles;
-  int S = (2 * ctx->sm_count) / (tiles > 0 ? tiles : 1);
+  // (measured: cluster launches place a little less than two CTAs per SM; asking for more than about
+  // 2 x SMs - 32 CTAs spills into a second wave)
+  int S = (2 * ctx->sm_count - 32) / (tiles > 0 ? tiles : 1);
   S = S < 1 ? 1 : (S > kMaxSplits ? kMaxSplits : S);
   if (S > G) S = G;
   const int forced = tc_env_int("ROSAQ_TC_SPLITS", 0);
