@@ -33,6 +33,7 @@ constexpr int kBoxBytes = 64 * kCovTokens * 2;          // one TMA box: 64 chann
 constexpr int kOperandBytes = 2 * kBoxBytes;            // 128 channels (operand A)
 constexpr int kStageBytes = 6 * kBoxBytes;              // A (2 boxes) and up to 256 channels of B (4 boxes)
 constexpr uint32_t kCovTmemCols = 256;
+constexpr int kCovDrainPolls = 1 << 16;                 // for work in flight when a CTA gives up (not the context's limit)
 
 struct CovParams {
   float *C;
@@ -179,7 +180,7 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
       if (ab.set()) {  // let loads already in flight land before the CTA goes away
         for (int back = 1; back <= kCovStages && back <= issued; ++back) {
           const int u = issued - back;
-          for (long long it = 0; it < p.wait_limit; ++it)
+          for (int it = 0; it < kCovDrainPolls; ++it)
             if (mbar_try_wait(bar_full + 8 * (u % kCovStages), (u / kCovStages) & 1)) break;
         }
       }
@@ -203,6 +204,10 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const CovParams p) {
         if (++idx == kCovStages) idx = 0, lap ^= 1u;
       }
       tc_commit(bar_d);
+      if (ab.set()) {  // MMAs already issued must retire before the tensor memory is given back
+        for (int it = 0; it < kCovDrainPolls; ++it)
+          if (mbar_try_wait(bar_d, 0)) break;
+      }
     }
   } else {
     // ---------------- epilogue: TMEM -> shared (transposable staging) -> C += tile, C^T += tile^T

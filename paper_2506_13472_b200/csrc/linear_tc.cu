@@ -36,6 +36,10 @@ constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels 
 constexpr int kTmemCols = 256;
 constexpr int kMaxProblems = 4;   // weights sharing one activation in a launch (q/k/v, gate/up)
 constexpr int kMaxSplits = 8;
+// polls (about a microsecond each) granted to work already in flight when a CTA gives up: unlike the
+// waits of the pipeline this bound does not follow the context's wait limit, so that a shortened limit
+// can never let a CTA retire under its own copies or MMAs
+constexpr int kDrainPolls = 1 << 16;
 
 struct TcParams {
   // up to kMaxProblems weights of identical geometry (d_in, bits, salient groups) that multiply the same
@@ -370,7 +374,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       if (ab.set()) {  // let copies already in flight land before the CTA goes away
         for (int back = 1; back <= p.NW && back <= uc; ++back) {
           const int u = uc - back;
-          for (long long it = 0; it < p.wait_limit; ++it)
+          for (int it = 0; it < kDrainPolls; ++it)
             if (mbar_try_wait(bar_w_full + 8 * (u % p.NW), (u / p.NW) & 1)) break;
         }
       }
@@ -394,7 +398,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       if (ab.set()) {
         for (int back = 1; back <= p.NA && back <= gc; ++back) {
           const int u = gc - back;
-          for (long long it = 0; it < p.wait_limit; ++it)
+          for (int it = 0; it < kDrainPolls; ++it)
             if (mbar_try_wait(bar_x_full + 8 * (u % p.NA), (u / p.NA) & 1)) break;
         }
       }
@@ -417,6 +421,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
         tc_commit(bar_empty + 8 * st);
       }
       tc_commit(bar_d_full);
+      if (ab.set()) {  // MMAs already issued must retire before the tensor memory is given back
+        for (int it = 0; it < kDrainPolls; ++it)
+          if (mbar_try_wait(bar_d_full, 0)) break;
+      }
     }
   } else {
     // ---------------- dequantisation warps: shared memory -> registers -> TMEM
@@ -485,7 +493,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
           tmem_st16(a_addr + 32 * hf + 16, &r[16]);
         }
       }
-      if (!ok) break;
+      if (!ok) {
+        tc_wait_st();                              // stores of earlier slices of this group
+        break;
+      }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_a_full + 8 * st);

@@ -232,3 +232,33 @@ def test_argument_errors_are_codes_not_faults(ctx):
         ctx.linear(torch.zeros((4, 128), dtype=torch.float16, device="cuda"), w)   # ldx < d_in
     assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
     assert ctx.last_status() == rb.ROSAQ_OK
+
+
+# --------------------------------------------------------------------------- bounded waits
+def test_expired_wait_is_reported_and_the_context_stays_usable(ctx):
+    """Failure detection without a GPU fault: with the wait limit cut to one poll, a wait that cannot be
+    satisfied in time (the Gram kernel's epilogue waiting for ~100 us of accumulation) gives up: the
+    kernel lets its copies and MMAs in flight finish, frees its tensor memory and returns, the status
+    word reports ROSAQ_ERR_TIMEOUT, and the same context then computes correct results again."""
+    c = H.config_tiny()
+    w = ctx.quantize(dev(c["W"]), dev(c["R32"]), bits=4, k_salient=128)
+    rot = ctx.rotation_create(dev(c["R16"]))
+    x = dev(c["x"])
+    want = ctx.linear(x, w, rot).cpu().numpy()
+    X = torch.randn((32768, 512), device="cuda").to(torch.float16)
+    Cg = torch.zeros((512, 512), dtype=torch.float32, device="cuda")
+    old = ctx.set_wait_limit(1)
+    try:
+        ctx.calib_cov(X, Cg)                                  # ~100 us of accumulation per tile
+        assert ctx.last_status() == rb.ROSAQ_ERR_TIMEOUT
+        assert ctx.last_status() == rb.ROSAQ_OK               # reading the status clears it
+    finally:
+        ctx.set_wait_limit(old)
+    got = ctx.linear(x, w, rot).cpu().numpy()
+    assert ctx.last_status() == rb.ROSAQ_OK
+    assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    Cg.zero_()
+    ctx.calib_cov(X[:1024], Cg)
+    assert ctx.last_status() == rb.ROSAQ_OK
+    Cref = X[:1024].double().T @ X[:1024].double()
+    assert torch.allclose(Cg.double(), Cref, rtol=1e-3, atol=1e-2)
