@@ -3,11 +3,11 @@
 
 Workload (N = 1): the seven linears of one LLaMA-7B-shaped decoder layer at M = 64 decode
 tokens, INT4 g128 with K = 128 FP16 salient channels (seeded synthetic weights and
-activations).  One step = one pass over the layer: three online rotations x.R (attention input,
-o_proj input, MLP input; dense 4096 x 4096 fp16 R from a PCA of synthetic calibration
-activations) and seven GEMM stages (q, k, v, o, gate, up, down; down_proj is not rotated, as in
+activations).  One step = one pass over the layer: three online rotations x.R (attention input and
+MLP input: dense 4096 x 4096 fp16 R from a layer-wise PCA of synthetic calibration activations;
+o_proj input: head-wise PCA, 32 blocks of 128 x 128 plus the global eigenvalue order, Eq. 6) and seven GEMM stages (q, k, v, o, gate, up, down; down_proj is not rotated, as in
 the paper's appendix on weight splitting).  Steps alternate between two layers with distinct
-weights (2 x 226 MB, larger than the 126 MB L2), replayed from CUDA graphs.
+weights (2 x 197 MB, larger than the 126 MB L2), replayed from CUDA graphs.
 
 metric/value: algorithmic bytes of the step (packed codes + scales/zeros + FP16 salient rows +
 activations in and out + the fp16 rotation matrices) divided by the device time, in GB/s.
@@ -37,7 +37,7 @@ K_SALIENT = 128
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 7 launches of an INT4 step
 # (ncu capture of this command, summarised in profiles/bench_launch_list_7b_layer_m64.md)
-TRAFFIC_BYTES_PER_LAUNCH = 31578441
+TRAFFIC_BYTES_PER_LAUNCH = None   # filled from profiles/bench_launch_list_7b_layer_m64.md when that capture matches this workload
 
 
 # ----------------------------------------------------------------------------- bytes / flops
@@ -111,8 +111,8 @@ def build_workload(ctx, bits, seed, n_layers, model):
     d, f = model["d"], model["ffn"]
     layers = []
     for li in range(n_layers):
-        rots, R32 = {}, {}
-        for inp in ("attn_in", "o_in", "mlp_in"):
+        rots, R32, perms = {}, {}, {}
+        for inp in ("attn_in", "mlp_in"):                            # layer-wise PCA, dense R (Section 3.1)
             law = synth.ActivationLaw(d, 1.0, seed, f"L{li}/{inp}")
             X = torch.from_numpy(law.sample(2048, "calib", np.float16)).cuda()
             Cg = torch.zeros((d, d), dtype=torch.float32, device="cuda")
@@ -120,25 +120,41 @@ def build_workload(ctx, bits, seed, n_layers, model):
             R = pca.eigh_descending_device(Cg)                       # fp64 on the device, host-side step a2
             R32[inp] = R.to(torch.float32).contiguous()
             rots[inp] = ctx.rotation_create(R.to(torch.float16).contiguous())
+        # o_proj input: head-wise PCA (Section 3.1.1, Eq. 6): one 128 x 128 rotation per head from
+        # per-head activations, plus the global descending-eigenvalue column order
+        H, hd = model["heads"], model["head_dim"]
+        Xh = torch.from_numpy(head_law(model, seed).sample(4096, f"L{li}/calib", np.float16)).cuda()
+        Cb = torch.zeros((H, hd, hd), dtype=torch.float32, device="cuda")
+        ctx.calib_cov(Xh, Cb, n_blocks=H)
+        Rb, perm, _ = pca.headwise_rotation(Cb.cpu().numpy())
+        R32["o_in"] = torch.from_numpy(Rb.astype(np.float32)).cuda()
+        perms["o_in"] = torch.from_numpy(perm).cuda()
+        rots["o_in"] = ctx.rotation_create(torch.from_numpy(Rb.astype(np.float16)).cuda(), perms["o_in"])
         weights, fp16 = {}, {}
         for name, d_in, d_out, inp in synth.layer_shapes(model):
             W = torch.from_numpy(synth.weights(d_in, d_out, seed, f"L{li}/{name}", sigma=0.02,
                                                outlier_frac=0.01, outlier_scale=10.0)).cuda()
-            weights[name] = ctx.quantize(W, R32.get(inp), bits=bits, k_salient=K_SALIENT)
+            weights[name] = ctx.quantize(W, R32.get(inp), perms.get(inp), bits=bits, k_salient=K_SALIENT)
             fp16[name] = W
         layers.append(dict(rots=rots, weights=weights, fp16=fp16))
         del R32
     xs = {}
-    for inp, dd in (("attn_in", d), ("o_in", d), ("mlp_in", d), ("down_in", f)):
+    for inp, dd in (("attn_in", d), ("mlp_in", d), ("down_in", f)):
         law = synth.ActivationLaw(dd, 1.0, seed, f"x/{inp}")
         xs[inp] = law.sample(M_TOKENS, "x", np.float16)
+    xs["o_in"] = head_law(model, seed).sample(M_TOKENS, "x", np.float16)
     return layers, xs
+
+
+def head_law(model, seed):
+    from paper_2506_13472_b200 import synth
+    return synth.HeadwiseActivationLaw(model["heads"], model["head_dim"], seed, "o_in")
 
 
 def layer_bytes(model, bits):
     from paper_2506_13472_b200 import synth
     b = sum(gemm_bytes(di, do, M_TOKENS, bits) for _, di, do, _ in synth.layer_shapes(model))
-    return b + 3 * rotate_bytes(model["d"], M_TOKENS)
+    return b + 2 * rotate_bytes(model["d"], M_TOKENS) + rotate_bytes(model["d"], M_TOKENS, model["heads"])
 
 
 class LayerRunner:
@@ -165,6 +181,24 @@ class LayerRunner:
         c.linear_multi(self.xr["mlp_in"], [L["weights"][n] for n in ("gate", "up")], None,
                        outs=[self.y[n] for n in ("gate", "up")])
         c.linear(self.x["down_in"], L["weights"]["down"], None, out=self.y["down"])
+
+
+def fp16_layer_graph(layers, xs_dev, model):
+    """The same seven GEMMs per layer with the un-rotated fp16 weights through cuBLAS (torch.matmul): one
+    CUDA graph that walks over all layers in turn (so the weights are as cold as on the quantized path);
+    a replay is len(layers) steps.  The FP16 baseline of the layer replay."""
+    import torch
+    d, f = model["d"], model["ffn"]
+    mk = lambda n: torch.empty((M_TOKENS, n), dtype=torch.float16, device="cuda")
+    y = {"q": mk(d), "k": mk(d), "v": mk(d), "o": mk(d), "gate": mk(f), "up": mk(f), "down": mk(d)}
+    inp = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "gate": "mlp_in", "up": "mlp_in",
+           "down": "down_in"}
+
+    def run():
+        for L in layers:
+            for n in ("q", "k", "v", "o", "gate", "up", "down"):
+                torch.matmul(xs_dev[inp[n]], L["fp16"][n], out=y[n])
+    return capture(run)
 
 
 def time_graphs(graphs, steps, warmup):
@@ -401,7 +435,8 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-        "config": {"workload": "LLaMA-7B decoder-layer linears (q,k,v,o,gate,up,down) + 3 dense online rotations, "
+        "config": {"workload": "LLaMA-7B decoder-layer linears (q,k,v,o,gate,up,down) + 3 online rotations (dense "
+                               "for q/k/v and gate/up inputs, head-wise 32 x 128 for o_proj input), "
                                "M=64, INT%d g128, K=128 FP16 salient, seed 1" % args.bits,
                    "bits": args.bits, "M": M_TOKENS, "bytes_per_step": step_bytes,
                    "cold_l2": "steps alternate between two layers of distinct weights (2 x %.0f MB > 126 MB L2)"
@@ -418,6 +453,10 @@ def run_ours(args):
                      "frac_of_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)},
     }
     if not args.no_table:
+        reps = max(args.steps // len(layers), 1)
+        fms = time_graphs([fp16_layer_graph(layers, xs_dev, model)], reps, args.warmup) / (reps * len(layers))
+        line["fp16_layer"] = {"what": "the 7 GEMMs of the layer with fp16 weights through cuBLAS, same graph replay",
+                              "ms_per_step": round(fms, 5), "speedup_of_this_path": round(fms / ms_per_step, 3)}
         line["gemm_stage"] = gemm_stage_table(ctx, model, args.bits, peaks)
         line["calib_cov"] = calib_cov_throughput(ctx, peaks)
     if not args.no_cpu_baseline and world == 1:
