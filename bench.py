@@ -37,7 +37,7 @@ K_SALIENT = 128
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 7 launches of an INT4 step
 # (ncu capture of this command, summarised in profiles/bench_launch_list_7b_layer_m64.md)
-TRAFFIC_BYTES_PER_LAUNCH = None   # filled from profiles/bench_launch_list_7b_layer_m64.md when that capture matches this workload
+TRAFFIC_BYTES_PER_LAUNCH = 26935223
 
 
 # ----------------------------------------------------------------------------- bytes / flops
