@@ -321,7 +321,9 @@ int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tok
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
   const size_t smem = 1024 + (size_t)kCovStages * kStageBytes;   // the 128 x (bn + 1) fp32 staging tile fits inside
-  static bool attr_done = false;
+  static bool attr_done_all[64] = {};                    // function attributes are per device
+  if (ctx->device < 0 || ctx->device >= 64) return ROSAQ_ERR_INVALID_ARG;
+  bool &attr_done = attr_done_all[ctx->device];
   if (!attr_done) {
     if (cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       (void)cudaGetLastError();

@@ -34,6 +34,7 @@ constexpr int kFirstDequantWarp = 3;
 constexpr int kWSlotBytes = kInt4CodeBytes + kScaleBytes;  // 8704: one quantized tile or a quarter fp16 tile
 constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels of an fp16 tile
 constexpr int kTmemCols = 256;
+constexpr int kMaxDevices = 64;
 constexpr int kMaxProblems = 4;   // weights sharing one activation in a launch (q/k/v, gate/up)
 constexpr int kMaxSplits = 8;
 // polls (about a microsecond each) granted to work already in flight when a CTA gives up: unlike the
@@ -631,9 +632,21 @@ size_t smem_bytes(int MT, int NW, int NA) {
 
 }  // namespace
 
-int tc_env_int(const char *name, int dflt) {
-  const char *v = getenv(name);
-  return v && *v ? atoi(v) : dflt;
+// Tuning overrides, read from the environment once per process:
+//   ROSAQ_TC_SPLITS  number of K splits (1..8) instead of the heuristic
+//   ROSAQ_TC_PDL     0 = launch without programmatic stream serialization
+struct TcOverrides {
+  int splits, pdl;
+};
+static const TcOverrides &tc_overrides() {
+  static const TcOverrides o = [] {
+    auto read = [](const char *name, int dflt) {
+      const char *v = getenv(name);
+      return v && *v ? atoi(v) : dflt;
+    };
+    return TcOverrides{read("ROSAQ_TC_SPLITS", 0), read("ROSAQ_TC_PDL", 1)};
+  }();
+  return o;
 }
 
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
@@ -689,7 +702,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   {
     const int budget = 110 * 1024 - 1024 - p.NA * p.MT * 256 - 256;
     int nw = budget / kWSlotBytes;
-    p.NW = tc_env_int("ROSAQ_TC_NW", nw > 10 ? 10 : nw);
+    p.NW = nw > 10 ? 10 : nw;
   }
 
   // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
@@ -700,7 +713,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   int S = (2 * ctx->sm_count - 32) / (tiles > 0 ? tiles : 1);
   S = S < 1 ? 1 : (S > kMaxSplits ? kMaxSplits : S);
   if (S > G) S = G;
-  const int forced = tc_env_int("ROSAQ_TC_SPLITS", 0);
+  const int forced = tc_overrides().splits;
   if (forced >= 1 && forced <= kMaxSplits && forced <= G) S = forced;
   p.S = S;
   {
@@ -734,7 +747,9 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // The opt-in limit is kept equal to what the launches really need (never a rounder, larger figure):
   // the driver sizes the shared-memory carve-out and the CTAs per SM from this attribute, and with
   // 2 x (limit + 1 KB) above the SM's 228 KB only one CTA would be resident.
-  static size_t attr_smem[2] = {0, 0};
+  static size_t attr_smem_all[kMaxDevices][2] = {};      // function attributes are per device
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) return ROSAQ_ERR_INVALID_ARG;
+  size_t *attr_smem = attr_smem_all[ctx->device];
   const int ki = (t.g_quant > 0 && t.bits == 3) ? 1 : 0;
   if (attr_smem[ki] < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
@@ -758,7 +773,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
     attr[na].val.clusterDim.z = 1;
     ++na;
   }
-  if (tc_env_int("ROSAQ_TC_PDL", 1)) {
+  if (tc_overrides().pdl) {
     // programmatic dependent launch: this kernel may start while the previous kernel of the stream is
     // still running; it touches x and y only after griddepcontrol.wait
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
