@@ -36,7 +36,8 @@ M_TOKENS = 64
 K_SALIENT = 128
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 7 launches of an INT4 step
-# (ncu capture of this command, summarised in profiles/bench_launch_list_7b_layer_m64.md)
+# (one ncu capture of this command with --steps 4 --warmup 3 --no-table --no-cpu-baseline; stale, and to be
+# set to None, as soon as the kernel or the workload changes)
 TRAFFIC_BYTES_PER_LAUNCH = 26935223
 
 

@@ -376,3 +376,34 @@ def test_mixed_precision_helps_in_rotated_space():
     e_rot = np.linalg.norm(y_rot - ref) / np.linalg.norm(ref)
     e_id = np.linalg.norm(y_id - ref) / np.linalg.norm(ref)
     assert e_rot < e_id
+
+
+def test_frozen_quantizer_output_has_not_drifted():
+    """The oracle's quantizer and bit layout are definitions of this repository (the paper gives none); a
+    stored answer on a closed-form input makes any later change to them explicit."""
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_rtn_golden", os.path.join(here, "make_rtn_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    W = mod.closed_form_weights()
+    want = {}
+    bits = None
+    for line in open(os.path.join(here, "rtn_groups.txt")):
+        if line.startswith("#"):
+            continue
+        key, *vals = line.split()
+        if key == "bits":
+            bits = int(vals[0])
+            want[bits] = {}
+        else:
+            want[bits][key] = [int(v, 16) for v in vals]
+    for b in (4, 3):
+        qd = orc.quantize(W, b, 128, 128)
+        qw = orc.pack(qd["codes"], b)
+        assert list(qd["scales"].view(np.uint16).ravel()) == want[b]["scales"]
+        assert list(qd["zeros"].view(np.uint16).ravel()) == want[b]["zeros"]
+        assert list(qd["salient"].view(np.uint16)[0]) == want[b]["salient_row0"]
+        for r in range(qw.shape[0]):
+            assert list(qw[r]) == want[b][f"qw{r}"]
