@@ -304,7 +304,7 @@ def profile_shape(args):
 def calib_cov_throughput(ctx, peaks, n_tokens=16384, d=5120, reps=5):
     """rosaq_calib_cov on one chunk of the 13B-shaped calibration stream (fp16 activations, fp32 C):
     device time per call and tensor throughput.  `tflops` counts the multiply-adds the kernel executes
-    (the 128 x 256 tiles that touch the lower triangle); `tflops_full_square` credits the
+    (the 256 x 256 tiles that touch the lower triangle); `tflops_full_square` credits the
     whole d x d result that those tiles produce by symmetry."""
     import torch
     X = torch.randn((n_tokens, d), device="cuda", dtype=torch.float16)
@@ -320,8 +320,8 @@ def calib_cov_throughput(ctx, peaks, n_tokens=16384, d=5120, reps=5):
         torch.cuda.synchronize()
         ts.append(e0.elapsed_time(e1))
     ms = sorted(ts)[len(ts) // 2]
-    nt = (d + 127) // 128                              # 128-row blocks; block bi has bi // 2 + 1 tiles of 128 x 256
-    executed = 2.0 * n_tokens * 128 * 256 * sum(bi // 2 + 1 for bi in range(nt))
+    nb = (d + 255) // 256                              # 256 x 256 tiles that touch the lower triangle
+    executed = 2.0 * n_tokens * 256 * 256 * (nb * (nb + 1) // 2)
     tf = executed / ms / 1e9
     return dict(tokens=n_tokens, d=d, ms=round(ms, 4), tflops=round(tf, 1),
                 tflops_full_square=round(2.0 * n_tokens * d * d / ms / 1e9, 1),
