@@ -89,7 +89,11 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
 
 /* Selects the rosaq_linear / rosaq_rotate implementation: 0 = tensor-core path
  * (tcgen05 + TMEM; default), 1 = plain CUDA-core path (slow; for debugging and
- * cross-checks -- it is still a GPU kernel of this library).  Returns the previous value. */
+ * cross-checks -- it is still a GPU kernel of this library), 2 = tensor-core path with
+ * CTA pairs (tcgen05 cta_group::2: two SMs share one MMA stream) wherever the shape allows
+ * it (token tile a multiple of 32, an even number of 128-column tiles); the K splits may
+ * differ from those of 0, so results agree to fp32 summation order, not bit for bit.
+ * Returns the previous value. */
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl);
 
 /* ---- calibration: Eq. 4, left-hand side ---------------------------------------- */

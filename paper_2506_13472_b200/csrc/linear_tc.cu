@@ -151,6 +151,62 @@ __device__ __forceinline__ void tc_mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uin
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster, ranks 2j and 2j + 1, drive one MMA stream
+template <uint32_t kCols>
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t holder_smem) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "n"(kCols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+template <uint32_t kCols>
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "n"(kCols) : "memory");
+}
+// commit whose arrival is delivered to the barrier at the same offset in every CTA of `mask`
+__device__ __forceinline__ void tc_commit_mc(uint32_t bar, uint32_t mask) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"((unsigned short)mask)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// load whose bytes are counted on a barrier of the pair's leader (a shared::cluster address); no multicast
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t lead_bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
+          "r"(dst),
+      "l"(map), "r"(lead_bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(1000u)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tc_mma8_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_lo, uint64_t b_hi,
+                                                uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %4, p;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 16;\n\tadd.u64 t, %2, 4;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 24;\n\tadd.u64 t, %2, 6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 32;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], %3, %4, q;\n\t"
+      "add.u32 a, %1, 40;\n\tadd.u64 t, %3, 2;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 48;\n\tadd.u64 t, %3, 4;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
+      "add.u32 a, %1, 56;\n\tadd.u64 t, %3, 6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
                "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
@@ -265,16 +321,20 @@ struct Abort {
   volatile int *flag;     // shared
   int *status;            // global
   long long limit;
+  bool cluster_scope;     // barriers also receive arrivals from the peer CTA of a pair
   __device__ __forceinline__ bool set() const { return *flag != 0; }
   __device__ __forceinline__ void raise() const {
     *flag = 1;
     atomicExch(status, (int)ROSAQ_ERR_TIMEOUT);
   }
   // false when the wait gave up (or somebody else already did)
+  __device__ __forceinline__ bool poll(uint32_t bar, uint32_t parity) const {
+    return cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
+  }
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (poll(bar, parity)) return true;
     for (long long it = 0; it < limit; ++it) {
-      if (mbar_try_wait(bar, parity)) return true;
+      if (poll(bar, parity)) return true;
       if ((it & 63) == 63 && set()) return false;
     }
     raise();
@@ -295,14 +355,19 @@ struct Ring {
   }
 };
 
-template <int kBits>
+// kPair: two CTAs with adjacent column tiles (cluster ranks 2j, 2j + 1; blockIdx.x even / odd) run as a
+// cta_group::2 pair.  Each dequantises its own 128 columns into its own tensor memory and loads half of
+// the token rows; the leader (even rank) issues one M = 256 MMA for both, so the per-SM cost of issuing
+// MMAs -- the bound of the single-CTA kernel at small token counts -- halves.
+template <int kBits, bool kPair>
 __global__ void __launch_bounds__(kThreads, 2)
 linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve-up (the dynamic window is 1024-byte aligned by the launch code's padding)
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int MT = p.MT;
-  const uint32_t x_slot_bytes = (uint32_t)MT * 256u;
+  const int MTL = kPair ? MT >> 1 : MT;                        // token rows this CTA keeps in shared memory
+  const uint32_t x_slot_bytes = (uint32_t)MTL * 256u;
   const uint32_t x_ring = base;                                // NA slots: one per TMEM operand buffer
   const uint32_t w_ring = x_ring + p.NA * x_slot_bytes;
   const uint32_t bars = w_ring + p.NW * kWSlotBytes;          // 8-byte aligned (all sizes multiples of 16)
@@ -323,7 +388,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   __half *const y_out = p.y[prob];
   const long long ldy = p.ldy[prob];
   const int g_begin = p.g_bounds[split], g_end = p.g_bounds[split + 1];
-  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit};
+  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit, kPair};
+  const uint32_t pair_x = kPair ? (blockIdx.x & 1u) : 0u;      // 0 = leader of the pair
+  const uint32_t lead_rank = kPair ? 2u * (uint32_t)split : 0u;   // cluster rank of this pair's leader
+  const bool is_lead = pair_x == 0;
+  const int n_arrive = kPair ? 2 * (kDequantThreads / 32) : kDequantThreads;   // arrivals that complete an a_full phase
 
   // Let the next kernel of the stream start its own prologue and weight prefetch while this one runs
   // (it only matters when the launches are chained programmatically; otherwise a no-op).
@@ -336,7 +405,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     }
     for (int i = 0; i < p.NA; ++i) {
       mbar_init(bar_x_full + 8 * i, 1);
-      mbar_init(bar_a_full + 8 * i, kDequantThreads);
+      mbar_init(bar_a_full + 8 * i, n_arrive);
       mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_d_full, 1);
@@ -344,9 +413,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 2) tmem_alloc<kTmemCols>(misc);
+  if (warp == 2) {
+    if (kPair) tmem_alloc_pair<kTmemCols>(misc);             // both CTAs of the pair, same warp index
+    else tmem_alloc<kTmemCols>(misc);
+  }
   tc_fence_before();
   __syncthreads();
+  if (kPair) {                                               // the peer's barriers and tensor memory exist
+    cluster_arrive();
+    cluster_wait();
+  }
   tc_fence_after();
   const uint32_t tmem = misc_ptr[0];
   const uint32_t a_col0 = (MT <= 64) ? 64u : 128u;             // A buffers follow the accumulator columns
@@ -392,24 +468,37 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
         const int slot = rs.idx;
         if (!ab.wait(bar_empty + 8 * slot, rs.lap ^ 1u)) break;
         const int k0 = (g_block0 + g) * kGroup;
-        mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
-        tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
-        tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
+        if (kPair) {
+          // each CTA loads its half of the token rows; all bytes are counted on the leader's barrier
+          if (is_lead) mbar_arrive_expect_tx(bar_x_full + 8 * slot, 2 * x_slot_bytes);
+          const uint32_t lb = map_to_rank(bar_x_full + 8 * slot, lead_rank);
+          const int mrow = m0 + (int)pair_x * MTL;
+          tma_load_2d_pair(x_ring + slot * x_slot_bytes, &xmap, lb, k0, mrow);
+          tma_load_2d_pair(x_ring + slot * x_slot_bytes + MTL * 128, &xmap, lb, k0 + 64, mrow);
+        } else {
+          mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
+          tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
+          tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
+        }
       }
-      if (ab.set()) {
+      // (in a pair the leader's barriers count the loads of both CTAs, and the peer stays until the
+      // cluster barrier at the end of the kernel, which the leader reaches after this drain)
+      if (ab.set() && is_lead) {
         for (int back = 1; back <= p.NA && back <= gc; ++back) {
           const int u = gc - back;
           for (int it = 0; it < kDrainPolls; ++it)
-            if (mbar_try_wait(bar_x_full + 8 * (u % p.NA), (u / p.NA) & 1)) break;
+            if (ab.poll(bar_x_full + 8 * (u % p.NA), (u / p.NA) & 1)) break;
         }
       }
     }
   } else if (warp == 2) {
     // ---------------- MMA issuer: per group one wait pair, eight MMAs, one commit
-    if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
+    if (lane == 0 && is_lead) {
+      // M = 128 output columns (256 for a pair), N = MT tokens
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | ((kPair ? 16u : 8u) << 24);
+      const uint32_t pair_mask = 3u << lead_rank;            // the two CTAs of the pair, for multicast commits
       const uint64_t desc0 = make_b_desc(x_ring);            // descriptor address fields are in 16-byte units
-      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MT * 128) >> 4;
+      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MTL * 128) >> 4;
       Ring rs{0, 0};
       uint32_t accumulate = 0;
       for (int g = g_begin; g < g_end; ++g, rs.advance(p.NA)) {
@@ -417,14 +506,20 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
         if (!ab.wait(bar_x_full + 8 * st, rs.lap) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
         tc_fence_after();
         const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
-        tc_mma8_ts(tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+        if (kPair) {
+          tc_mma8_ts_pair(tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+          tc_commit_mc(bar_empty + 8 * st, pair_mask);
+        } else {
+          tc_mma8_ts(tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+          tc_commit(bar_empty + 8 * st);
+        }
         accumulate = 1;
-        tc_commit(bar_empty + 8 * st);
       }
-      tc_commit(bar_d_full);
+      if (kPair) tc_commit_mc(bar_d_full, pair_mask);
+      else tc_commit(bar_d_full);
       if (ab.set()) {  // MMAs already issued must retire before the tensor memory is given back
         for (int it = 0; it < kDrainPolls; ++it)
-          if (mbar_try_wait(bar_d_full, 0)) break;
+          if (ab.poll(bar_d_full, 0)) break;
       }
     }
   } else {
@@ -500,7 +595,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_a_full + 8 * st);
+      if (kPair) {
+        // one arrival per warp, on the leader's barrier
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_a_full + 8 * st, lead_rank));
+      } else {
+        mbar_arrive(bar_a_full + 8 * st);
+      }
     }
   }
 
@@ -542,7 +643,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       }
     }
   } else {
-    const uint32_t rank = cluster_rank();
+    const uint32_t rank = (uint32_t)split;                   // the K split of this CTA owns token rows rank, rank + S, ...
     const int rows_max = (MT + p.S - 1) / p.S;               // rows any rank can own
     const uint32_t recv = base;                              // [source rank][row slot][128] fp32
     cluster_arrive();                                        // #1: this CTA no longer touches its rings
@@ -557,7 +658,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const uint32_t dst = recv + (uint32_t)(((int)rank * rows_max + jrow) * kTileN + n) * 4u;
-          st_cluster_u32(map_to_rank(dst, (uint32_t)r), v[e]);
+          st_cluster_u32(map_to_rank(dst, kPair ? 2u * (uint32_t)r + pair_x : (uint32_t)r), v[e]);
           if (++r == p.S) {
             r = 0;
             ++jrow;
@@ -596,9 +697,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
 
   tc_fence_before();
   __syncthreads();
+  if (kPair && p.S == 1) {                                   // the pair gives its tensor memory back together
+    cluster_arrive();
+    cluster_wait();
+  }
   if (warp == 2) {
     __syncwarp();
-    tmem_dealloc<kTmemCols>(tmem);
+    if (kPair) tmem_dealloc_pair<kTmemCols>(tmem);
+    else tmem_dealloc<kTmemCols>(tmem);
   }
 }
 
@@ -699,8 +805,15 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // stages (TMEM operand buffer + activation slot of MT x 128 channels): 3 next to 64 accumulator
   // columns, 2 next to 128; the rest of a half SM's shared memory goes to the packed-weight ring
   p.NA = p.MT <= 64 ? 3 : 2;
+  // CTA pairs: adjacent column tiles of one weight, token count a multiple of 32 (MMA N of a pair)
+  // (a block-diagonal operand pairs up only if both tiles of a pair multiply the same channels)
+  // Off unless asked for (linear implementation 2): on the decode shapes measured so far the pair's
+  // cross-CTA handshakes cost more than the halved MMA issue saves.
+  bool pair = ctx->impl == 2 && p.MT % 32 == 0 && t.block_groups % 2 == 0;
+  for (int i = 0; i < n && pair; ++i) pair = ts[i]->n_tiles % 2 == 0;
+  const int MTL = pair ? p.MT / 2 : p.MT;                  // token rows a CTA keeps in shared memory
   {
-    const int budget = 110 * 1024 - 1024 - p.NA * p.MT * 256 - 256;
+    const int budget = 110 * 1024 - 1024 - p.NA * MTL * 256 - 256;
     int nw = budget / kWSlotBytes;
     p.NW = nw > 10 ? 10 : nw;
   }
@@ -711,10 +824,11 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // (measured: cluster launches place a little less than two CTAs per SM; asking for more than about
   // 2 x SMs - 32 CTAs spills into a second wave)
   int S = (2 * ctx->sm_count - 32) / (tiles > 0 ? tiles : 1);
-  S = S < 1 ? 1 : (S > kMaxSplits ? kMaxSplits : S);
+  const int max_splits = pair ? kMaxSplits / 2 : kMaxSplits;    // a cluster holds the S splits of both CTAs of a pair
+  S = S < 1 ? 1 : (S > max_splits ? max_splits : S);
   if (S > G) S = G;
   const int forced = tc_overrides().splits;
-  if (forced >= 1 && forced <= kMaxSplits && forced <= G) S = forced;
+  if (forced >= 1 && forced <= max_splits && forced <= G) S = forced;
   p.S = S;
   {
     // cost(g) = 4 for an fp16 group, 1 for a quantized one; bound sp is the first group whose
@@ -734,7 +848,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   {
     const cuuint64_t dims[2] = {(cuuint64_t)t.d_in, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
-    const cuuint32_t box[2] = {64, (cuuint32_t)p.MT};
+    const cuuint32_t box[2] = {64, (cuuint32_t)MTL};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(x), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -742,15 +856,17 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
     if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
   }
 
-  const size_t smem = smem_bytes(p.MT, p.NW, p.NA);
-  auto kern = (t.g_quant > 0 && t.bits == 3) ? linear_tc_kernel<3> : linear_tc_kernel<4>;
+  const size_t smem = smem_bytes(MTL, p.NW, p.NA);
+  const bool int3 = t.g_quant > 0 && t.bits == 3;
+  auto kern = pair ? (int3 ? linear_tc_kernel<3, true> : linear_tc_kernel<4, true>)
+                   : (int3 ? linear_tc_kernel<3, false> : linear_tc_kernel<4, false>);
   // The opt-in limit is kept equal to what the launches really need (never a rounder, larger figure):
   // the driver sizes the shared-memory carve-out and the CTAs per SM from this attribute, and with
   // 2 x (limit + 1 KB) above the SM's 228 KB only one CTA would be resident.
-  static size_t attr_smem_all[kMaxDevices][2] = {};      // function attributes are per device
+  static size_t attr_smem_all[kMaxDevices][4] = {};      // function attributes are per device
   if (ctx->device < 0 || ctx->device >= kMaxDevices) return ROSAQ_ERR_INVALID_ARG;
   size_t *attr_smem = attr_smem_all[ctx->device];
-  const int ki = (t.g_quant > 0 && t.bits == 3) ? 1 : 0;
+  const int ki = (int3 ? 1 : 0) + (pair ? 2 : 0);
   if (attr_smem[ki] < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -766,9 +882,9 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   int na = 0;
-  if (S > 1) {
+  if (S > 1 || pair) {
     attr[na].id = cudaLaunchAttributeClusterDimension;
-    attr[na].val.clusterDim.x = 1;
+    attr[na].val.clusterDim.x = pair ? 2 : 1;
     attr[na].val.clusterDim.y = S;
     attr[na].val.clusterDim.z = 1;
     ++na;

@@ -160,7 +160,7 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
   if (!ctx) return 0;
   int prev = ctx->impl;
-  if (impl == 0 || impl == 1) ctx->impl = impl;
+  if (impl >= 0 && impl <= 2) ctx->impl = impl;
   return prev;
 }
 

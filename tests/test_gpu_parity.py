@@ -165,6 +165,30 @@ def test_linear_multi_gives_the_bits_of_separate_calls(ctx, bits, M):
     assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("M,d_in,d_out,k_salient", [(64, 1024, 512, 128), (128, 512, 256, 128), (32, 2048, 256, 0),
+                                                      (200, 512, 512, 256)])
+def test_linear_cta_pairs_give_the_bits_of_single_ctas(ctx, M, d_in, d_out, k_salient, bits):
+    """Implementation 2 (two CTAs per MMA stream, cta_group::2) on shapes it accepts: within the oracle
+    tolerance, and equal to the default implementation up to the fp32 summation order of the K splits."""
+    W = synth.weights(d_in, d_out, seed=61, key=f"pair{d_in}x{d_out}", outlier_frac=0.01)
+    x = synth.rng_for(61, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+    R = H.config_tiny()["R16"] if d_in == 512 else None
+    w = ctx.quantize(dev(W), None, bits=bits, k_salient=k_salient)
+    rot = None if R is None else ctx.rotation_create(dev(R))
+    qd = H.oracle_quantized(W, None, None, bits, k_salient)
+    want = ctx.linear(dev(x), w, rot).cpu().numpy()
+    ctx.set_linear_impl(2)
+    try:
+        got = ctx.linear(dev(x), w, rot).cpu().numpy()
+        check_status(ctx)
+    finally:
+        ctx.set_linear_impl(0)
+    assert np.all(np.isfinite(got))
+    assert H.rel_fro(got, want) <= 2e-4
+    assert H.rel_fro(got, orc.forward(x, qd, R)) <= H.REL_TOL_Y
+
+
 def test_special_case_all_salient_is_plain_fp16_gemm(ctx):
     rng = np.random.default_rng(12)
     W = (rng.standard_normal((256, 128)) * 0.02).astype(np.float16)
