@@ -331,6 +331,22 @@ struct Abort {
   __device__ __forceinline__ bool poll(uint32_t bar, uint32_t parity) const {
     return cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
   }
+  // barriers that only this CTA's threads and copies feed: CTA scope whatever the mode
+  __device__ __forceinline__ bool wait_local(uint32_t bar, uint32_t parity) const {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (long long it = 0; it < limit; ++it) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((it & 63) == 63 && set()) return false;
+    }
+    raise();
+    return false;
+  }
+  // one cluster-scope poll per warp instead of thirty-two, verdict broadcast (also the warp-level sync)
+  __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity) const {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = wait(bar, parity) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+  }
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
     if (poll(bar, parity)) return true;
     for (long long it = 0; it < limit; ++it) {
@@ -443,7 +459,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
         const uint32_t bytes = f16 ? kFp16SubBytes : qbytes;
         for (int sub = 0; sub < nsub; ++sub, ++uc, rw.advance(p.NW)) {
           const int slot = rw.idx;
-          if (!ab.wait(bar_w_empty + 8 * slot, rw.lap ^ 1u)) break;
+          if (!ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u)) break;
           mbar_arrive_expect_tx(bar_w_full + 8 * slot, bytes);
           bulk_copy_g2s(w_ring + slot * kWSlotBytes, src + (long long)sub * kFp16SubBytes, bytes, bar_w_full + 8 * slot);
         }
@@ -536,10 +552,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       const int nsub = f16 ? 4 : 1;
       const int st = rs.idx;
       const uint32_t a_addr = lane_addr + a_col0 + st * 64;
-      bool got = ab.wait(bar_empty + 8 * st, rs.lap ^ 1u);
+      bool got = kPair ? ab.wait_warp(bar_empty + 8 * st, rs.lap ^ 1u) : ab.wait(bar_empty + 8 * st, rs.lap ^ 1u);
       for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(p.NW)) {
         const int slot = rw.idx;
-        got = got && ab.wait(bar_w_full + 8 * slot, rw.lap);
+        got = got && ab.wait_local(bar_w_full + 8 * slot, rw.lap);
         got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
         if (!got) {
           ok = false;
