@@ -30,7 +30,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "rosaq_w4a16_decode_layer_hbm_gbs_m64"
+METRIC = "rosaq_w4a16_decode_layer_hbm_gbs_m64"     # "w3" when run with --bits 3
 UNIT = "GB/s"
 M_TOKENS = 64
 K_SALIENT = 128
@@ -365,7 +365,7 @@ def run_reference(args):
         vals.append(v)
     v = float(np.mean(vals))
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": METRIC.replace("w4", "w%d" % args.bits), "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": None, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "7B decoder-layer linears, M=64, INT%d g128 K=128 (oracle on a column sample)" % args.bits},
@@ -433,7 +433,7 @@ def run_ours(args):
         return
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC.replace("w4", "w%d" % args.bits), "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
         "config": {"workload": "LLaMA-7B decoder-layer linears (q,k,v,o,gate,up,down) + 3 online rotations (dense "
