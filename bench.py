@@ -356,17 +356,19 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    vals = []
+    vals, t_steps = [], []
     for _ in range(args.warmup):
         oracle_sample(args.bits, seconds_hint=1.0)
     text, cores = "", 1
     for _ in range(args.steps):
+        t0 = time.perf_counter()
         v, cores, text = oracle_sample(args.bits, seconds_hint=max(2.0, 60.0 / max(args.steps, 1)))
+        t_steps.append(time.perf_counter() - t0)
         vals.append(v)
     v = float(np.mean(vals))
     print(json.dumps({
         "impl": "reference", "metric": METRIC.replace("w4", "w%d" % args.bits), "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": None, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": round(1e3 * float(np.mean(t_steps)), 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "7B decoder-layer linears, M=64, INT%d g128 K=128 (oracle on a column sample)" % args.bits},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": text},
