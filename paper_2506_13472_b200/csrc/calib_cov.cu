@@ -255,29 +255,59 @@ cov_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ 
       float *Cb = p.C + (long long)h * p.dh * p.dh;
       const int i0 = bi * kCovTile, j0 = bj * p.bn;
       // C[i0 + r][j0 + c] += tile[r][c]: a warp touches 32 consecutive floats of one row of C
-      // (eight independent loads in flight per thread before the adds: the update is latency-bound)
-      const int n_rows = min(kCovTile, p.dh - i0), n_cols = min(p.bn, p.dh - j0);
-      for (int c = tid; c < n_cols; c += 128) {
-        float *dst = Cb + (long long)i0 * p.dh + j0 + c;
-        for (int r0 = 0; r0 < n_rows; r0 += 8) {
-          float old[8];
+      // The update of C is latency-bound (read-modify-write through L2), so each thread keeps eight
+      // independent 16-byte loads in flight.  Direct part: C[i0 + r][j0 + 4 q .. + 3] += tile[r][4 q .. + 3].
+      const int n_rows = min(kCovTile, p.dh - i0), n_cols = min(p.bn, p.dh - j0);   // both multiples of 8
+      {
+        const int quads = p.bn >> 2, sets = 128 / quads;   // 64 x 2 or 32 x 4 (column quads x interleaved row sets)
+        const int q = tid % quads, r_first = tid / quads;
+        if (4 * q < n_cols) {
+          float *dst = Cb + (long long)i0 * p.dh + j0 + 4 * q;
+          for (int r0 = r_first; r0 < n_rows; r0 += 8 * sets) {
+            float4 old[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) old[e] = r0 + e < n_rows ? __ldcg(dst + (long long)(r0 + e) * p.dh) : 0.0f;
+            for (int e = 0; e < 8; ++e) {
+              const int r = r0 + sets * e;
+              old[e] = r < n_rows ? __ldcg(reinterpret_cast<const float4 *>(dst + (long long)r * p.dh))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (r0 + e < n_rows) dst[(long long)(r0 + e) * p.dh] = __fadd_rn(old[e], stage[(r0 + e) * pitch + c]);
+            for (int e = 0; e < 8; ++e) {
+              const int r = r0 + sets * e;
+              if (r < n_rows) {
+                const float *t = stage + r * pitch + 4 * q;
+                *reinterpret_cast<float4 *>(dst + (long long)r * p.dh) =
+                    make_float4(__fadd_rn(old[e].x, t[0]), __fadd_rn(old[e].y, t[1]), __fadd_rn(old[e].z, t[2]),
+                                __fadd_rn(old[e].w, t[3]));
+              }
+            }
+          }
         }
       }
-      // mirror: C[j0 + c][i0 + tid] += tile[tid][c]
-      if (!diag && tid < n_rows) {
-        float *dst = Cb + (long long)j0 * p.dh + i0 + tid;
-        for (int c0 = 0; c0 < n_cols; c0 += 8) {
-          float old[8];
+      // mirror: C[j0 + c][i0 + 4 q .. + 3] += tile[4 q .. + 3][c]
+      if (!diag) {
+        const int q = tid & 31, c_first = tid >> 5;       // 32 row quads of the tile x 4 interleaved column sets
+        if (4 * q < n_rows) {
+          float *dst = Cb + (long long)j0 * p.dh + i0 + 4 * q;
+          for (int c0 = c_first; c0 < n_cols; c0 += 32) {
+            float4 old[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) old[e] = c0 + e < n_cols ? __ldcg(dst + (long long)(c0 + e) * p.dh) : 0.0f;
+            for (int e = 0; e < 8; ++e) {
+              const int c = c0 + 4 * e;
+              old[e] = c < n_cols ? __ldcg(reinterpret_cast<const float4 *>(dst + (long long)c * p.dh))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (c0 + e < n_cols) dst[(long long)(c0 + e) * p.dh] = __fadd_rn(old[e], stage[tid * pitch + c0 + e]);
+            for (int e = 0; e < 8; ++e) {
+              const int c = c0 + 4 * e;
+              if (c < n_cols) {
+                const float *t = stage + (4 * q) * pitch + c;
+                *reinterpret_cast<float4 *>(dst + (long long)c * p.dh) =
+                    make_float4(__fadd_rn(old[e].x, t[0]), __fadd_rn(old[e].y, t[pitch]), __fadd_rn(old[e].z, t[2 * pitch]),
+                                __fadd_rn(old[e].w, t[3 * pitch]));
+              }
+            }
+          }
         }
       }
     }
