@@ -30,6 +30,7 @@ namespace {
 
 constexpr int kThreads = 352;
 constexpr int kDequantThreads = 256;
+constexpr int kTeamThreads = 128;                          // one dequantisation team: a warp per TMEM lane quadrant
 constexpr int kFirstDequantWarp = 3;
 constexpr int kWSlotBytes = kInt4CodeBytes + kScaleBytes;  // 8704: one quantized tile or a quarter fp16 tile
 constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels of an fp16 tile
@@ -206,11 +207,6 @@ __device__ __forceinline__ void tc_mma8_ts_pair(uint32_t d_tmem, uint32_t a_tmem
       "add.u32 a, %1, 56;\n\tadd.u64 t, %3, 6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
-               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
   asm volatile(
@@ -408,7 +404,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const uint32_t pair_x = kPair ? (blockIdx.x & 1u) : 0u;      // 0 = leader of the pair
   const uint32_t lead_rank = kPair ? 2u * (uint32_t)split : 0u;   // cluster rank of this pair's leader
   const bool is_lead = pair_x == 0;
-  const int n_arrive = kPair ? 2 * (kDequantThreads / 32) : kDequantThreads;   // arrivals that complete an a_full phase
+  const int n_arrive = kPair ? 2 * (kTeamThreads / 32) : kTeamThreads;   // arrivals that complete an a_full phase
 
   // Let the next kernel of the stream start its own prologue and weight prefetch while this one runs
   // (it only matters when the launches are chained programmatically; otherwise a no-op).
@@ -417,7 +413,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.NW; ++i) {
       mbar_init(bar_w_full + 8 * i, 1);
-      mbar_init(bar_w_empty + 8 * i, kDequantThreads);
+      mbar_init(bar_w_empty + 8 * i, kTeamThreads);
     }
     for (int i = 0; i < p.NA; ++i) {
       mbar_init(bar_x_full + 8 * i, 1);
@@ -540,9 +536,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     }
   } else {
     // ---------------- dequantisation warps: shared memory -> registers -> TMEM
+    // Two teams of four warps (one warp per TMEM lane quadrant) take alternate groups, so that the
+    // waits, the TMEM store drain and the barrier traffic of one team run under the arithmetic of the
+    // other; a thread dequantises all 128 input channels of its output column.
     const int dq = warp - kFirstDequantWarp;       // 0..7
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may touch
-    const int hf = dq >> 2;                        // which half of the slot's K range
+    const int team = dq >> 2;
     const int n = quad * 32 + lane;                // output column inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     Ring rw{0, 0}, rs{0, 0};
@@ -550,59 +549,61 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     for (int g = g_begin; g < g_end && ok; ++g, rs.advance(p.NA)) {
       const bool f16 = g < p.g_fp16;
       const int nsub = f16 ? 4 : 1;
+      if (((g - g_begin) & 1) != team) {           // the other team's group: only keep the ring positions
+        for (int sub = 0; sub < nsub; ++sub) rw.advance(p.NW);
+        continue;
+      }
       const int st = rs.idx;
       const uint32_t a_addr = lane_addr + a_col0 + st * 64;
       bool got = kPair ? ab.wait_warp(bar_empty + 8 * st, rs.lap ^ 1u) : ab.wait(bar_empty + 8 * st, rs.lap ^ 1u);
       for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(p.NW)) {
         const int slot = rw.idx;
-        got = got && ab.wait_local(bar_w_full + 8 * slot, rw.lap);
+        // A parity wait must not be a whole phase early.  The previous fill of this slot may belong to
+        // the other team, which can lag by a group: first see that fill released (the same phase the
+        // producer waits for), only then wait for the new one.
+        got = got && ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u) && ab.wait_local(bar_w_full + 8 * slot, rw.lap);
         got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
         if (!got) {
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t ws = w_ring + slot * kWSlotBytes;
+        const uint32_t ws = w_ring + slot * kWSlotBytes + n * 16;
         if (f16) {
-          // a quarter of an fp16 group: 32 input channels = 16 TMEM columns, 8 per half
-          uint32_t r[8];
-          *reinterpret_cast<uint4 *>(&r[0]) = lds128(ws + ((2 * hf + 0) * kTileN + n) * 16);
-          *reinterpret_cast<uint4 *>(&r[4]) = lds128(ws + ((2 * hf + 1) * kTileN + n) * 16);
+          // a quarter of an fp16 group: 32 input channels = 16 TMEM columns
+          uint32_t r[16];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4 *>(&r[4 * j]) = lds128(ws + j * (kTileN * 16));
           mbar_arrive(bar_w_empty + 8 * slot);
-          tmem_st8(a_addr + 16 * sub + 8 * hf, r);
+          tmem_st16(a_addr + 16 * sub, r);
         } else if (kBits == 4) {
-          const ScaleZero c(lds32(ws + kInt4CodeBytes + n * 4));
-          const uint4 q0 = lds128(ws + ((2 * hf + 0) * kTileN + n) * 16);
-          const uint4 q1 = lds128(ws + ((2 * hf + 1) * kTileN + n) * 16);
+          const ScaleZero c(lds32(w_ring + slot * kWSlotBytes + kInt4CodeBytes + n * 4));
+          uint4 q[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) q[j] = lds128(ws + j * (kTileN * 16));
           mbar_arrive(bar_w_empty + 8 * slot);
-          uint32_t r[32];
-          dequant_int4_word(q0.x, c, &r[0]);
-          dequant_int4_word(q0.y, c, &r[4]);
-          dequant_int4_word(q0.z, c, &r[8]);
-          dequant_int4_word(q0.w, c, &r[12]);
-          tmem_st16(a_addr + 32 * hf, &r[0]);
-          dequant_int4_word(q1.x, c, &r[16]);
-          dequant_int4_word(q1.y, c, &r[20]);
-          dequant_int4_word(q1.z, c, &r[24]);
-          dequant_int4_word(q1.w, c, &r[28]);
-          tmem_st16(a_addr + 32 * hf + 16, &r[16]);
-        } else {
-          const ScaleZero c(lds32(ws + kInt3CodeBytes + n * 4));
-          // this half needs words 6*hf .. 6*hf+5 of the column's 12: chunks hf and hf+1
-          const uint4 qa = lds128(ws + ((hf + 0) * kTileN + n) * 16);
-          const uint4 qb = lds128(ws + ((hf + 1) * kTileN + n) * 16);
-          mbar_arrive(bar_w_empty + 8 * slot);
-          uint32_t w6[6];
-          if (hf == 0) {
-            w6[0] = qa.x, w6[1] = qa.y, w6[2] = qa.z, w6[3] = qa.w, w6[4] = qb.x, w6[5] = qb.y;
-          } else {
-            w6[0] = qa.z, w6[1] = qa.w, w6[2] = qb.x, w6[3] = qb.y, w6[4] = qb.z, w6[5] = qb.w;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t r[16];
+            dequant_int4_word(q[j].x, c, &r[0]);
+            dequant_int4_word(q[j].y, c, &r[4]);
+            dequant_int4_word(q[j].z, c, &r[8]);
+            dequant_int4_word(q[j].w, c, &r[12]);
+            tmem_st16(a_addr + 16 * j, r);
           }
-          uint32_t r[32];
-          dequant_int3_set(w6[0], w6[1], w6[2], c, &r[0]);
-          tmem_st16(a_addr + 32 * hf, &r[0]);
-          dequant_int3_set(w6[3], w6[4], w6[5], c, &r[16]);
-          tmem_st16(a_addr + 32 * hf + 16, &r[16]);
+        } else {
+          const ScaleZero c(lds32(w_ring + slot * kWSlotBytes + kInt3CodeBytes + n * 4));
+          // the column's 12 words: 4 sets of 3 words = 32 codes = 16 TMEM columns each
+          uint32_t w12[12];
+#pragma unroll
+          for (int j = 0; j < 3; ++j) *reinterpret_cast<uint4 *>(&w12[4 * j]) = lds128(ws + j * (kTileN * 16));
+          mbar_arrive(bar_w_empty + 8 * slot);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t r[16];
+            dequant_int3_set(w12[3 * j], w12[3 * j + 1], w12[3 * j + 2], c, r);
+            tmem_st16(a_addr + 16 * j, r);
+          }
         }
       }
       if (!ok) {
