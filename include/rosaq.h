@@ -92,7 +92,11 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
  * cross-checks -- it is still a GPU kernel of this library), 2 = tensor-core path with
  * CTA pairs (tcgen05 cta_group::2: two SMs share one MMA stream) wherever the shape allows
  * it (token tile a multiple of 32, an even number of 128-column tiles); the K splits may
- * differ from those of 0, so results agree to fp32 summation order, not bit for bit.
+ * differ from those of 0, so results agree to fp32 summation order, not bit for bit;
+ * 3 = tensor-core path that always splits K across thread-block clusters (0 prefers,
+ * for token counts up to 64 and operands with enough column tiles, an equal share of the
+ * weight stream per SM with the partial tiles exchanged through a workspace that
+ * rosaq_create allocated; again the same sums in another order).
  * Returns the previous value. */
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl);
 

@@ -312,6 +312,53 @@ __device__ __forceinline__ void dequant_int3_set(uint32_t a, uint32_t b, uint32_
   out[15] = h2_sub_mul(tail | 0x64006400u, c.z1024, c.s2);
 }
 
+// One unit of the weight ring (a quantized group, or 32 input channels of an fp16 group) of output
+// column n: shared memory -> registers -> the TMEM operand buffer at a_addr.  The slot is released
+// only after instructions that depend on every loaded word have been issued: an arrive placed right
+// behind the loads can be performed while they are still queued (seen when the other CTA of the SM kept
+// the load/store unit busy with global stores), and the producer then refills the slot under them.
+template <int kBits>
+__device__ __forceinline__ void dequant_unit(bool f16, uint32_t slot_base, int n, uint32_t a_addr, int sub,
+                                             uint32_t bar_release) {
+  const uint32_t ws = slot_base + n * 16;
+  if (f16) {
+    // a quarter of an fp16 group: 32 input channels = 16 TMEM columns
+    uint32_t r[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4 *>(&r[4 * j]) = lds128(ws + j * (kTileN * 16));
+    tmem_st16(a_addr + 16 * sub, r);
+    mbar_arrive(bar_release);
+  } else if (kBits == 4) {
+    const ScaleZero c(lds32(slot_base + kInt4CodeBytes + n * 4));
+    uint4 q[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) q[j] = lds128(ws + j * (kTileN * 16));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t r[16];
+      dequant_int4_word(q[j].x, c, &r[0]);
+      dequant_int4_word(q[j].y, c, &r[4]);
+      dequant_int4_word(q[j].z, c, &r[8]);
+      dequant_int4_word(q[j].w, c, &r[12]);
+      tmem_st16(a_addr + 16 * j, r);
+    }
+    mbar_arrive(bar_release);
+  } else {
+    const ScaleZero c(lds32(slot_base + kInt3CodeBytes + n * 4));
+    // the column's 12 words: 4 sets of 3 words = 32 codes = 16 TMEM columns each
+    uint32_t w12[12];
+#pragma unroll
+    for (int j = 0; j < 3; ++j) *reinterpret_cast<uint4 *>(&w12[4 * j]) = lds128(ws + j * (kTileN * 16));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t r[16];
+      dequant_int3_set(w12[3 * j], w12[3 * j + 1], w12[3 * j + 2], c, r);
+      tmem_st16(a_addr + 16 * j, r);
+    }
+    mbar_arrive(bar_release);
+  }
+}
+
 // ---------------------------------------------------------------------------------- the kernel
 struct Abort {
   volatile int *flag;     // shared
@@ -568,43 +615,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
           break;
         }
         tc_fence_after();
-        const uint32_t ws = w_ring + slot * kWSlotBytes + n * 16;
-        if (f16) {
-          // a quarter of an fp16 group: 32 input channels = 16 TMEM columns
-          uint32_t r[16];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4 *>(&r[4 * j]) = lds128(ws + j * (kTileN * 16));
-          mbar_arrive(bar_w_empty + 8 * slot);
-          tmem_st16(a_addr + 16 * sub, r);
-        } else if (kBits == 4) {
-          const ScaleZero c(lds32(w_ring + slot * kWSlotBytes + kInt4CodeBytes + n * 4));
-          uint4 q[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) q[j] = lds128(ws + j * (kTileN * 16));
-          mbar_arrive(bar_w_empty + 8 * slot);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t r[16];
-            dequant_int4_word(q[j].x, c, &r[0]);
-            dequant_int4_word(q[j].y, c, &r[4]);
-            dequant_int4_word(q[j].z, c, &r[8]);
-            dequant_int4_word(q[j].w, c, &r[12]);
-            tmem_st16(a_addr + 16 * j, r);
-          }
-        } else {
-          const ScaleZero c(lds32(w_ring + slot * kWSlotBytes + kInt3CodeBytes + n * 4));
-          // the column's 12 words: 4 sets of 3 words = 32 codes = 16 TMEM columns each
-          uint32_t w12[12];
-#pragma unroll
-          for (int j = 0; j < 3; ++j) *reinterpret_cast<uint4 *>(&w12[4 * j]) = lds128(ws + j * (kTileN * 16));
-          mbar_arrive(bar_w_empty + 8 * slot);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t r[16];
-            dequant_int3_set(w12[3 * j], w12[3 * j + 1], w12[3 * j + 2], c, r);
-            tmem_st16(a_addr + 16 * j, r);
-          }
-        }
+        dequant_unit<kBits>(f16, w_ring + slot * kWSlotBytes, n, a_addr, sub, bar_w_empty + 8 * slot);
       }
       if (!ok) {
         tc_wait_st();                              // stores of earlier slices of this group
@@ -725,6 +736,354 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------------- stream-K variant
+// For token tiles of at most 64 tokens and operands with enough column tiles, the (tile, group) list of
+// the whole launch is cut into one contiguous range per CTA (two CTAs per SM, equal cost), so every SM
+// streams the same number of bytes whatever the tile count.  A range covers the tail of one tile and the
+// head of the next at most: two accumulators in tensor memory, one main loop over both, one epilogue.
+// A tile shared by several CTAs is finished by the one that holds its last groups: the others store
+// their fp32 partial tile to a workspace and count themselves in; the finisher waits for them (they all
+// have lower block indices, hence were dispatched before it), adds the partials in ascending K order
+// and its own accumulator last, and writes y.  The sum order is fixed, so results are reproducible.
+constexpr int kMaxSkCtas = kSkMaxCtas;
+constexpr int kSkStages = 2;                       // one TMEM operand buffer + activation slot per team
+constexpr int kSkTokens = 64;                      // token capacity of an accumulator and of a partial tile
+
+struct SkParams {
+  int n_prob;
+  int tile_start[kMaxProblems + 1];
+  const uint8_t *blob[kMaxProblems];
+  int d_out[kMaxProblems];
+  __half *y[kMaxProblems];
+  long long ldy[kMaxProblems];
+  long long tile_stride;
+  int g_fp16, g_quant, block_groups;
+  int G;                     // groups per tile
+  int M, MT;
+  int NW;
+  const int32_t *col_map;
+  int *status;
+  long long wait_limit;
+  float *partials;           // [CTA][2][64 tokens][128 columns]
+  int *arrive;               // [tile]: partial tiles stored so far; zero between launches
+  int bounds[kMaxSkCtas + 1];   // CTA i owns entries [bounds[i], bounds[i + 1]) of the tile-major (tile, group) list
+};
+
+struct SkTile {
+  int prob, nt;
+  const uint8_t *base;
+};
+
+__device__ __forceinline__ SkTile sk_tile(const SkParams &p, int tile) {
+  int prob = 0;
+  while (prob + 1 < p.n_prob && tile >= p.tile_start[prob + 1]) ++prob;
+  const int nt = tile - p.tile_start[prob];
+  return SkTile{prob, nt, p.blob[prob] + (long long)nt * p.tile_stride};
+}
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire(const int *ptr) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+template <int kBits>
+__global__ void __launch_bounds__(kThreads, 2)
+linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ SkParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int MT = p.MT;
+  const uint32_t x_slot_bytes = (uint32_t)MT * 256u;
+  const uint32_t x_ring = base;
+  const uint32_t w_ring = x_ring + kSkStages * x_slot_bytes;
+  const uint32_t bars = w_ring + p.NW * kWSlotBytes;
+  const uint32_t bar_w_full = bars, bar_w_empty = bar_w_full + 8 * p.NW;
+  const uint32_t bar_x_full = bar_w_empty + 8 * p.NW, bar_a_full = bar_x_full + 8 * kSkStages;
+  const uint32_t bar_empty = bar_a_full + 8 * kSkStages;
+  const uint32_t bar_d_full = bar_empty + 8 * kSkStages;       // two: one per accumulator
+  const uint32_t misc = bar_d_full + 16;                       // [0] TMEM base, [1] abort flag
+  uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t *misc_ptr = reinterpret_cast<volatile uint32_t *>(gen + (misc - base));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  const int u_begin = p.bounds[cta], n_units = p.bounds[cta + 1] - u_begin;
+  const int tile0 = u_begin / p.G, g0 = u_begin - tile0 * p.G;
+  const int len0 = n_units < p.G - g0 ? n_units : p.G - g0;    // entries of the first tile; the rest start the next tile
+  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit, false};
+
+  grid_dep_launch_dependents();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.NW; ++i) {
+      mbar_init(bar_w_full + 8 * i, 1);
+      mbar_init(bar_w_empty + 8 * i, kTeamThreads);
+    }
+    for (int i = 0; i < kSkStages; ++i) {
+      mbar_init(bar_x_full + 8 * i, 1);
+      mbar_init(bar_a_full + 8 * i, kTeamThreads);
+      mbar_init(bar_empty + 8 * i, 1);
+      mbar_init(bar_d_full + 8 * i, 1);
+    }
+    misc_ptr[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) tmem_alloc<kTmemCols>(misc);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc_ptr[0];
+  // columns: accumulator of the first tile at 0, of the second at 64, operand buffers at 128 and 192
+  const uint32_t a_col0 = 2 * kSkTokens;
+  const int qbytes = quant_tile_bytes(kBits);
+
+  if (warp == 0) {
+    // ---------------- weight-tile producer
+    if (lane == 0) {
+      int uc = 0;
+      Ring rw{0, 0};
+      int tile = tile0, g = g0;
+      const uint8_t *tile_base = sk_tile(p, tile).base;
+      for (int j = 0; j < n_units && !ab.set(); ++j) {
+        const bool f16 = g < p.g_fp16;
+        const uint8_t *src = tile_base + (f16 ? (long long)g * kFp16TileBytes
+                                              : (long long)p.g_fp16 * kFp16TileBytes + (long long)(g - p.g_fp16) * qbytes);
+        const int nsub = f16 ? 4 : 1;
+        const uint32_t bytes = f16 ? kFp16SubBytes : qbytes;
+        bool live = true;
+        for (int sub = 0; sub < nsub; ++sub, ++uc, rw.advance(p.NW)) {
+          const int slot = rw.idx;
+          if (!ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u)) {
+            live = false;
+            break;
+          }
+          mbar_arrive_expect_tx(bar_w_full + 8 * slot, bytes);
+          bulk_copy_g2s(w_ring + slot * kWSlotBytes, src + (long long)sub * kFp16SubBytes, bytes, bar_w_full + 8 * slot);
+        }
+        if (!live) break;
+        if (++g == p.G && j + 1 < n_units) {
+          g = 0;
+          tile_base = sk_tile(p, ++tile).base;
+        }
+      }
+      if (ab.set()) {  // let copies already in flight land before the CTA goes away
+        for (int back = 1; back <= p.NW && back <= uc; ++back) {
+          const int u = uc - back;
+          for (int it = 0; it < kDrainPolls; ++it)
+            if (mbar_try_wait(bar_w_full + 8 * (u % p.NW), (u / p.NW) & 1)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- activation producer
+    if (lane == 0) {
+      grid_dep_wait();                                         // x may be the previous kernel's output
+      int gc = 0;
+      Ring rs{0, 0};
+      int tile = tile0, g = g0;
+      auto block0 = [&](int t) {
+        const int nt = sk_tile(p, t).nt;
+        return p.block_groups > 0 ? (nt / p.block_groups) * p.block_groups : 0;
+      };
+      int g_block0 = block0(tile);
+      for (int j = 0; j < n_units && !ab.set(); ++j, ++gc, rs.advance(kSkStages)) {
+        const int slot = rs.idx;
+        if (!ab.wait(bar_empty + 8 * slot, rs.lap ^ 1u)) break;
+        const int k0 = (g_block0 + g) * kGroup;
+        mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
+        tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, 0);
+        tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, 0);
+        if (++g == p.G && j + 1 < n_units) {
+          g = 0;
+          g_block0 = block0(++tile);
+        }
+      }
+      if (ab.set()) {
+        for (int back = 1; back <= kSkStages && back <= gc; ++back) {
+          const int u = gc - back;
+          for (int it = 0; it < kDrainPolls; ++it)
+            if (mbar_try_wait(bar_x_full + 8 * (u % kSkStages), (u / kSkStages) & 1)) break;
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
+      const uint64_t desc0 = make_b_desc(x_ring);
+      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MT * 128) >> 4;
+      Ring rs{0, 0};
+      uint32_t accumulate = 0;
+      int g = g0, seg = 0, committed = 0;
+      for (int j = 0; j < n_units; ++j, rs.advance(kSkStages)) {
+        const int st = rs.idx;
+        if (!ab.wait(bar_x_full + 8 * st, rs.lap) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
+        tc_fence_after();
+        const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
+        tc_mma8_ts(tmem + seg * kSkTokens, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+        tc_commit(bar_empty + 8 * st);
+        accumulate = 1;
+        if (++g == p.G || j + 1 == n_units) {                  // this tile's share is complete
+          tc_commit(bar_d_full + 8 * seg);
+          ++seg, ++committed;
+          g = 0;
+          accumulate = 0;
+        }
+      }
+      if (ab.set()) {  // MMAs already issued must retire before the tensor memory is given back
+        const uint32_t bar = bar_d_full + 8 * (committed < 2 ? committed : 1);
+        if (committed < 2) tc_commit(bar);
+        for (int it = 0; it < kDrainPolls; ++it)
+          if (mbar_try_wait(bar, 0)) break;
+      }
+    }
+  } else {
+    // ---------------- dequantisation: two teams on alternate entries, team = stage
+    const int dq = warp - kFirstDequantWarp;
+    const int quad = warp & 3;
+    const int team = dq >> 2;
+    const int n = quad * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    Ring rw{0, 0}, rs{0, 0};
+    bool ok = true;
+    int g = g0;
+    for (int j = 0; j < n_units && ok; ++j, rs.advance(kSkStages)) {
+      const bool f16 = g < p.g_fp16;
+      const int nsub = f16 ? 4 : 1;
+      if (++g == p.G) g = 0;
+      if ((j & 1) != team) {
+        for (int sub = 0; sub < nsub; ++sub) rw.advance(p.NW);
+        continue;
+      }
+      const int st = rs.idx;
+      const uint32_t a_addr = lane_addr + a_col0 + st * 64;
+      bool got = ab.wait(bar_empty + 8 * st, rs.lap ^ 1u);
+      for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(p.NW)) {
+        const int slot = rw.idx;
+        // first see the slot's previous fill released (it may belong to the other team, which can lag by
+        // an entry), then wait for the new one: a parity wait must not be a whole phase early
+        got = got && ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u) && ab.wait_local(bar_w_full + 8 * slot, rw.lap);
+        got = __all_sync(0xffffffffu, got);
+        if (!got) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        dequant_unit<kBits>(f16, w_ring + slot * kWSlotBytes, n, a_addr, sub, bar_w_empty + 8 * slot);
+      }
+      tc_wait_st();
+      if (!ok) break;
+      tc_fence_before();
+      mbar_arrive(bar_a_full + 8 * st);
+    }
+  }
+
+  // ---------------- epilogue: one pass per tile this CTA touched
+  // Thread (column n = TMEM lane, half hf of the tokens) owns tokens col0 .. col0 + MT/2 - 1 of column n.
+  const bool is_epi = warp >= kFirstDequantWarp;
+  if (is_epi) {
+    const int quad = warp & 3, hf = (warp - kFirstDequantWarp) >> 2;
+    const int n = quad * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    const int half_cols = MT >> 1, col0 = hf * half_cols;
+    const bool lead = threadIdx.x == kFirstDequantWarp * 32;
+    grid_dep_wait();                       // y, the partial tiles and the counters may still be in use by the previous kernel
+    const int n_seg = len0 < n_units ? 2 : 1;
+    // the second tile first: its partial tile waits for nobody, while finishing the first tile may wait
+    for (int seg = n_seg - 1; seg >= 0; --seg) {
+      const int tile = tile0 + seg;
+      const int gs = seg == 0 ? g0 : 0, len = seg == 0 ? len0 : n_units - len0;
+      bool have_d = ab.wait(bar_d_full + 8 * seg, 0);
+      have_d = __all_sync(0xffffffffu, have_d && !ab.set());
+      if (have_d) tc_fence_after();
+      const SkTile tr = sk_tile(p, tile);
+      const int d_out = p.d_out[tr.prob];
+      __half *const y_out = p.y[tr.prob];
+      const long long ldy = p.ldy[tr.prob];
+      const uint32_t d_addr = lane_addr + seg * kSkTokens + col0;
+      const bool finisher = gs + len == p.G;                   // holds the tile's last groups
+      if (!finisher) {
+        // store the partial tile [token][column] (a warp writes 128 contiguous bytes per token) and
+        // count this CTA in
+        if (have_d) {
+          uint32_t *dst = reinterpret_cast<uint32_t *>(p.partials) + (((long long)cta * 2 + seg) * kSkTokens + col0) * kTileN + n;
+          for (int c0 = 0; c0 < half_cols; c0 += 8) {
+            uint32_t v[8];
+            tmem_ld8(d_addr + c0, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dst[(c0 + e) * kTileN] = v[e];
+          }
+          __threadfence();
+        }
+        epi_bar();
+        if (lead && !ab.set()) atomicAdd(p.arrive + tile, 1);
+        continue;
+      }
+      // the finisher: contributors cf .. cta - 1 hold the earlier groups of this tile
+      int cf = cta;
+      while (cf > 0 && p.bounds[cf] > tile * p.G) --cf;
+      const int k_lower = cta - cf;
+      if (k_lower > 0) {
+        if (lead) {
+          bool seen = false;
+          for (long long it = 0; it < p.wait_limit && !seen; ++it) {
+            seen = ld_acquire(p.arrive + tile) >= k_lower;
+            if (!seen && (it & 63) == 63 && ab.set()) break;
+          }
+          if (!seen && !ab.set()) ab.raise();
+        }
+        epi_bar();
+        have_d = have_d && !ab.set();
+      }
+      if (have_d) {
+        const int n_glob = tr.nt * kTileN + n;
+        const bool n_ok = n_glob < d_out;
+        const long long out_col = n_ok ? (p.col_map ? p.col_map[n_glob] : n_glob) : 0;
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+        for (int c = cf; c < cta; ++c) {                       // ascending K; up to 32 coalesced loads in flight
+          const int slot = (c == cf && p.bounds[cf] < tile * p.G) ? 1 : 0;   // the tile is that CTA's second one
+          const float *src = p.partials + (((long long)c * 2 + slot) * kSkTokens + col0) * kTileN + n;
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = e < half_cols ? __ldcg(src + e * kTileN) : 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[e] += v[e];
+        }
+#pragma unroll
+        for (int c0 = 0; c0 < 32; c0 += 8) {
+          if (c0 < half_cols) {
+            uint32_t v[8];
+            tmem_ld8(d_addr + c0, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float r = acc[c0 + e] + __uint_as_float(v[e]);
+              const int mg = col0 + c0 + e;
+              if (n_ok && mg < p.M) y_out[(long long)mg * ldy + out_col] = __float2half_rn(r);
+            }
+          }
+        }
+      }
+      if (k_lower > 0) {
+        epi_bar();                                             // every thread has read the partial tiles
+        if (lead && !ab.set()) p.arrive[tile] = 0;             // ready for the next launch
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    __syncwarp();
+    tmem_dealloc<kTmemCols>(tmem);
+  }
+}
+
 // ---------------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -753,13 +1112,38 @@ size_t smem_bytes(int MT, int NW, int NA) {
   return b < 80 * 1024 ? 80 * 1024 : b;
 }
 
+
+size_t sk_smem_bytes(int MT, int NW) {
+  size_t b = 1024 + (size_t)kSkStages * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NW + 4 * kSkStages) + 16;
+  return b < 80 * 1024 ? 80 * 1024 : b;
+}
+
+// Cuts the tile-major (tile, group) list into P ranges of equal cost (an fp16 group weighs four quantized
+// ones), every cut on a group boundary.  False when a range would be empty or touch more than two tiles.
+bool sk_bounds(int T, int G, int g_fp16, int P, int *bounds) {
+  const long long C = 4ll * g_fp16 + (G - g_fp16), N = C * T;
+  for (int i = 0; i <= P; ++i) {
+    const long long c = N * i / P;
+    const long long tile = c / C, within = c % C;
+    const long long g = within < 4ll * g_fp16 ? within / 4 : g_fp16 + (within - 4ll * g_fp16);
+    bounds[i] = (int)(tile * G + g);
+  }
+  bounds[P] = T * G;
+  for (int i = 0; i < P; ++i) {
+    if (bounds[i + 1] <= bounds[i]) return false;
+    if ((bounds[i + 1] - 1) / G - bounds[i] / G > 1) return false;
+  }
+  return true;
+}
+
 }  // namespace
 
 // Tuning overrides, read from the environment once per process:
 //   ROSAQ_TC_SPLITS  number of K splits (1..8) instead of the heuristic
 //   ROSAQ_TC_PDL     0 = launch without programmatic stream serialization
+//   ROSAQ_TC_SK      0 = never use the stream-K variant; n > 1 = use it when CTAs <= n x column tiles
 struct TcOverrides {
-  int splits, pdl;
+  int splits, pdl, sk;
 };
 static const TcOverrides &tc_overrides() {
   static const TcOverrides o = [] {
@@ -767,9 +1151,60 @@ static const TcOverrides &tc_overrides() {
       const char *v = getenv(name);
       return v && *v ? atoi(v) : dflt;
     };
-    return TcOverrides{read("ROSAQ_TC_SPLITS", 0), read("ROSAQ_TC_PDL", 1)};
+    return TcOverrides{read("ROSAQ_TC_SPLITS", 0), read("ROSAQ_TC_PDL", 1), read("ROSAQ_TC_SK", 2)};
   }();
   return o;
+}
+
+static int launch_linear_sk(const rosaq_ctx *ctx, const __half *x, long long ldx, const TiledOperand &t, const SkParams &q,
+                            int P, cudaStream_t s) {
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return ROSAQ_ERR_CUDA;
+  CUtensorMap xmap;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)t.d_in, (cuuint64_t)q.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)q.MT};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(x), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
+  }
+  const size_t smem = sk_smem_bytes(q.MT, q.NW);
+  const bool int3 = t.g_quant > 0 && t.bits == 3;
+  auto kern = int3 ? linear_sk_kernel<3> : linear_sk_kernel<4>;
+  static size_t attr_smem_all[kMaxDevices][2] = {};       // function attributes are per device
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) return ROSAQ_ERR_INVALID_ARG;
+  size_t *attr_smem = attr_smem_all[ctx->device];
+  if (attr_smem[int3 ? 1 : 0] < smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return ROSAQ_ERR_CUDA;
+    }
+    attr_smem[int3 ? 1 : 0] = smem;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(P, 1, 1);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  int na = 0;
+  if (tc_overrides().pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, xmap, q);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
+  return ROSAQ_OK;
 }
 
 int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t,
@@ -828,6 +1263,32 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // cross-CTA handshakes cost more than the halved MMA issue saves.
   bool pair = ctx->impl == 2 && p.MT % 32 == 0 && t.block_groups % 2 == 0;
   for (int i = 0; i < n && pair; ++i) pair = ts[i]->n_tiles % 2 == 0;
+  // stream-K variant: token tile of at most 64 tokens, one token tile, and so many column tiles that a tile
+  // is shared by two or three CTAs at most (its finisher reads the others' partial tiles one after the
+  // other; measured at 64 tokens: 4096 -> 22016, 172 tiles, 24.1 us against 28.4 with cluster splits;
+  // with 96 tiles equal, with 86 tiles 1.7 us slower)
+  if (ctx->impl == 0 && !pair && m_tiles == 1 && p.MT <= kSkTokens && ctx->sk_partials && tc_overrides().sk > 0) {
+    const int P = ctx->sk_ctas < 2 * ctx->sm_count ? ctx->sk_ctas : 2 * ctx->sm_count;
+    if (n_tiles_all <= P && n_tiles_all <= kSkCounterInts && (long long)n_tiles_all * tc_overrides().sk >= P) {
+      SkParams q{};
+      if (sk_bounds(n_tiles_all, G, t.g_fp16, P, q.bounds)) {
+        q.n_prob = n;
+        for (int i = 0; i <= n; ++i) q.tile_start[i] = p.tile_start[i];
+        for (int i = 0; i < n; ++i) q.blob[i] = p.blob[i], q.d_out[i] = p.d_out[i], q.y[i] = p.y[i], q.ldy[i] = p.ldy[i];
+        q.tile_stride = p.tile_stride;
+        q.g_fp16 = p.g_fp16, q.g_quant = p.g_quant, q.block_groups = p.block_groups;
+        q.G = G, q.M = M, q.MT = p.MT;
+        q.col_map = col_map, q.status = p.status, q.wait_limit = p.wait_limit;
+        q.partials = ctx->sk_partials, q.arrive = ctx->sk_arrive;
+        {
+          const int budget = 110 * 1024 - 1024 - kSkStages * p.MT * 256 - 256;
+          const int nw = budget / kWSlotBytes;
+          q.NW = nw > 10 ? 10 : nw;
+        }
+        return launch_linear_sk(ctx, x, ldx, t, q, P, s);
+      }
+    }
+  }
   const int MTL = pair ? p.MT / 2 : p.MT;                  // token rows a CTA keeps in shared memory
   {
     const int budget = 110 * 1024 - 1024 - p.NA * MTL * 256 - 256;

@@ -109,10 +109,20 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->ws_bytes = 0;
   ctx->wait_limit = 1ll << 20;
   ctx->impl = 0;
+  ctx->sk_partials = nullptr;
+  ctx->sk_arrive = nullptr;
+  ctx->sk_ctas = 2 * ctx->sm_count < rosaq::kSkMaxCtas ? 2 * ctx->sm_count : rosaq::kSkMaxCtas;
   st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), sizeof(int)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
+  // the stream-K workspace is taken here, once, so that no linear call ever allocates for it
+  if (st == ROSAQ_OK)
+    st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->sk_partials), (size_t)ctx->sk_ctas * 2 * rosaq::kSkPartialBytes));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->sk_arrive), rosaq::kSkCounterInts * sizeof(int)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
   if (st != ROSAQ_OK) {
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
+    if (ctx->sk_arrive) (void)cudaFree(ctx->sk_arrive);
     delete ctx;
     return st;
   }
@@ -127,6 +137,8 @@ int rosaq_destroy(rosaq_ctx *ctx) {
     (void)cudaDeviceSynchronize();
     if (ctx->ws) (void)cudaFree(ctx->ws);
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
+    if (ctx->sk_arrive) (void)cudaFree(ctx->sk_arrive);
     (void)cudaGetLastError();
   }
   delete ctx;
@@ -146,6 +158,9 @@ int rosaq_last_status(rosaq_ctx *ctx, void *stream) {
   if (host != 0) {
     st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
     if (st != ROSAQ_OK) return st;
+    // a launch that gave up may have left arrival counters of the stream-K exchange behind
+    st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
+    if (st != ROSAQ_OK) return st;
   }
   return host;
 }
@@ -160,7 +175,7 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
   if (!ctx) return 0;
   int prev = ctx->impl;
-  if (impl >= 0 && impl <= 2) ctx->impl = impl;
+  if (impl >= 0 && impl <= 3) ctx->impl = impl;
   return prev;
 }
 

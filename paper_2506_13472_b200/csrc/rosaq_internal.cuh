@@ -163,6 +163,12 @@ __device__ __forceinline__ void load_quant_tile_column(const uint8_t *tile, int 
 // ---- handles -----------------------------------------------------------------------------
 }  // namespace rosaq
 
+namespace rosaq {
+constexpr int kSkMaxCtas = 320;                     // stream-K grid limit (two CTAs per SM)
+constexpr int kSkCounterInts = 1024;                // arrival counters (one per column tile of a launch)
+constexpr size_t kSkPartialBytes = 128 * 64 * sizeof(float);   // one partial tile: 128 columns x 64 tokens
+}  // namespace rosaq
+
 struct rosaq_ctx {
   int device;
   int sm_count;
@@ -170,7 +176,10 @@ struct rosaq_ctx {
   void *ws;            // rotated-activation workspace
   size_t ws_bytes;
   long long wait_limit;
-  int impl;            // 0 tensor-core, 1 CUDA-core
+  int impl;            // 0 tensor-core, 1 CUDA-core, 2 tensor-core with CTA pairs, 3 tensor-core without stream-K
+  float *sk_partials;  // stream-K: fp32 partial tiles, [sk_ctas][2][64 tokens][128 columns]
+  int *sk_arrive;      // stream-K: per-tile arrival counters, zero between launches
+  int sk_ctas;         // CTAs the partial-tile workspace was sized for
 };
 
 struct rosaq_weight {

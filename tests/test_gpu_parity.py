@@ -189,6 +189,56 @@ def test_linear_cta_pairs_give_the_bits_of_single_ctas(ctx, M, d_in, d_out, k_sa
     assert H.rel_fro(got, orc.forward(x, qd, R)) <= H.REL_TOL_Y
 
 
+
+# --------------------------------------------------------------------------- equal-share (stream-K) launches
+@pytest.mark.parametrize("bits", [4, 3])
+def test_linear_stream_k_path(ctx, bits):
+    """At up to 64 tokens an operand with at least as many column tiles as SMs is cut into equal shares of
+    the (tile, group) list, one per CTA, and tiles shared by several CTAs are finished through a workspace
+    (implementation 0); implementation 3 always splits K across clusters.  Both must match the oracle on
+    sampled columns; they agree up to the fp32 summation order; repeated launches give the same bits."""
+    d_in, d_out = 1024, 150 * 128
+    W = synth.weights(d_in, d_out, seed=71, key=f"sk{bits}", outlier_frac=0.01)
+    cols = synth.sample_columns(d_out, 24, 71, f"sk{bits}")
+    w = ctx.quantize(dev(W), None, bits=bits, k_salient=128)
+    qd = H.oracle_quantized(W, None, None, bits, 128, cols=cols)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    for M in (1, 16, 64):
+        x = synth.rng_for(71, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+        got = ctx.linear(dev(x), w, None).cpu().numpy()
+        again = ctx.linear(dev(x), w, None).cpu().numpy()
+        ctx.set_linear_impl(3)
+        try:
+            want = ctx.linear(dev(x), w, None).cpu().numpy()
+        finally:
+            ctx.set_linear_impl(0)
+        check_status(ctx)
+        assert np.all(np.isfinite(got))
+        assert np.array_equal(got.view(np.uint16), again.view(np.uint16))
+        assert H.rel_fro(got, want) <= 2e-4
+        assert H.rel_fro(got[:, cols], orc.forward(x, qd, None)) <= H.REL_TOL_Y
+    w.free()
+
+
+def test_linear_multi_stream_k_path(ctx):
+    """Two weights whose column tiles together fill the equal-share launch (gate/up style), against the
+    separate calls (which split K across clusters) and the oracle."""
+    d_in, d_out, M = 1024, 75 * 128, 64
+    Ws = [synth.weights(d_in, d_out, seed=72, key=f"skm{i}", outlier_frac=0.01) for i in range(2)]
+    ws = [ctx.quantize(dev(W), None, bits=4, k_salient=128) for W in Ws]
+    x = synth.rng_for(72, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+    want = [ctx.linear(dev(x), w, None).cpu().numpy() for w in ws]
+    got = [g.cpu().numpy() for g in ctx.linear_multi(dev(x), ws, None)]
+    check_status(ctx)
+    for i in range(2):
+        cols = synth.sample_columns(d_out, 16, 72, f"skm{i}")
+        qd = H.oracle_quantized(Ws[i], None, None, 4, 128, cols=cols)
+        assert H.rel_fro(got[i], want[i]) <= 2e-4
+        assert H.rel_fro(got[i][:, cols], orc.forward(x, qd, None)) <= H.REL_TOL_Y
+    for w in ws:
+        w.free()
+
+
 def test_special_case_all_salient_is_plain_fp16_gemm(ctx):
     rng = np.random.default_rng(12)
     W = (rng.standard_normal((256, 128)) * 0.02).astype(np.float16)
