@@ -38,7 +38,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 7 launches of an INT4 step
 # (one ncu capture of this command with --steps 4 --warmup 3 --no-table --no-cpu-baseline; stale, and to be
 # set to None, as soon as the kernel or the workload changes)
-TRAFFIC_BYTES_PER_LAUNCH = 26935223
+TRAFFIC_BYTES_PER_LAUNCH = 26943431
 
 
 # ----------------------------------------------------------------------------- bytes / flops
@@ -452,7 +452,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / peaks["hbm_gbs"], 4),
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.bits == 4 else None,
-                     "peak_source": peaks["source"], "kernel": "linear_tc_kernel<4> (all 7 launches of a step: 3 rotations, qkv, o, gate+up, down)",
+                     "peak_source": peaks["source"], "kernel": "linear_tc_kernel / linear_sk_kernel (all 7 launches of a step: 3 rotations, qkv, o, gate+up, down)",
                      "frac_of_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)},
     }
     if not args.no_table:

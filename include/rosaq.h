@@ -71,8 +71,12 @@ typedef struct {
 /* ---- context ---------------------------------------------------------------- */
 
 /* Creates a context on CUDA device `device` (must be compute capability 10.x, else
- * ROSAQ_ERR_UNSUPPORTED_ARCH).  Allocates a small device status word and, lazily,
- * a workspace for the rotated activations.  Synchronous. */
+ * ROSAQ_ERR_UNSUPPORTED_ARCH).  Allocates a small device status word, the workspace
+ * through which the CTAs of one rosaq_linear launch exchange partial output tiles
+ * (64 KB per CTA of a two-CTAs-per-SM grid, 19 MB on a 148-SM device, plus 4 KB of
+ * counters) and, lazily at the first call that needs it, a workspace for the rotated
+ * activations.  A context serves one stream at a time: calls on different streams
+ * that overlap in time need a context each.  Synchronous. */
 int rosaq_create(rosaq_ctx **out, int device);
 int rosaq_destroy(rosaq_ctx *ctx);
 
