@@ -38,6 +38,10 @@ constexpr int kTmemCols = 256;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxProblems = 4;   // weights sharing one activation in a launch (q/k/v, gate/up)
 constexpr int kMaxSplits = 8;
+// Relative cost of a group when work is divided: an fp16 group is 3.7 times the bytes of an INT4 group,
+// but up to 64 tokens a CTA is paced by its eight MMAs and its handshakes per group, not by bytes
+// (measured: weights 4 : 1 lose 2-5 % against 1.5 : 1 on the 7B shapes).
+constexpr int kCostFp16 = 3, kCostQuant = 2;
 // polls (about a microsecond each) granted to work already in flight when a CTA gives up: unlike the
 // waits of the pipeline this bound does not follow the context's wait limit, so that a shortened limit
 // can never let a CTA retire under its own copies or MMAs
@@ -1016,10 +1020,12 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
 #pragma unroll
             for (int e = 0; e < 8; ++e) dst[(c0 + e) * kTileN] = v[e];
           }
-          __threadfence();
         }
-        epi_bar();
-        if (lead && !ab.set()) atomicAdd(p.arrive + tile, 1);
+        epi_bar();                                             // all stores of the CTA are issued ...
+        if (lead && !ab.set()) {
+          __threadfence();                                     // ... and ordered before the count (cumulative fence)
+          atomicAdd(p.arrive + tile, 1);
+        }
         continue;
       }
       // the finisher: contributors cf .. cta - 1 hold the earlier groups of this tile
@@ -1118,14 +1124,14 @@ size_t sk_smem_bytes(int MT, int NW) {
   return b < 80 * 1024 ? 80 * 1024 : b;
 }
 
-// Cuts the tile-major (tile, group) list into P ranges of equal cost (an fp16 group weighs four quantized
-// ones), every cut on a group boundary.  False when a range would be empty or touch more than two tiles.
+// Cuts the tile-major (tile, group) list into P ranges of equal cost, every cut on a group boundary.  False when a range would be empty or touch more than two tiles.
 bool sk_bounds(int T, int G, int g_fp16, int P, int *bounds) {
-  const long long C = 4ll * g_fp16 + (G - g_fp16), N = C * T;
+  const long long FW = kCostFp16, QW = kCostQuant;
+  const long long C = FW * g_fp16 + QW * (G - g_fp16), N = C * T;
   for (int i = 0; i <= P; ++i) {
     const long long c = N * i / P;
     const long long tile = c / C, within = c % C;
-    const long long g = within < 4ll * g_fp16 ? within / 4 : g_fp16 + (within - 4ll * g_fp16);
+    const long long g = within < FW * g_fp16 ? within / FW : g_fp16 + (within - FW * g_fp16) / QW;
     bounds[i] = (int)(tile * G + g);
   }
   bounds[P] = T * G;
@@ -1297,21 +1303,25 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   }
 
   // K splits: fill about two CTAs per SM; each split gets a contiguous range of groups of roughly
-  // equal bytes (an fp16 group weighs four quantized ones)
+  // equal cost
   const int tiles = n_tiles_all * m_tiles;
   // (measured: cluster launches place a little less than two CTAs per SM; asking for more than about
   // 2 x SMs - 32 CTAs spills into a second wave)
   int S = (2 * ctx->sm_count - 32) / (tiles > 0 ? tiles : 1);
   const int max_splits = pair ? kMaxSplits / 2 : kMaxSplits;    // a cluster holds the S splits of both CTAs of a pair
-  S = S < 1 ? 1 : (S > max_splits ? max_splits : S);
+  // (six splits measured faster than eight on the 32-tile shapes: the exchange grows with the cluster)
+  const int auto_cap = pair ? max_splits : 6;
+  S = S < 1 ? 1 : (S > auto_cap ? auto_cap : S);
   if (S > G) S = G;
   const int forced = tc_overrides().splits;
   if (forced >= 1 && forced <= max_splits && forced <= G) S = forced;
   p.S = S;
   {
-    // cost(g) = 4 for an fp16 group, 1 for a quantized one; bound sp is the first group whose
+    // bound sp is the first group whose
     // preceding cost reaches sp/S of the total, clamped so that every range keeps a group
-    auto cost_before = [&](int g) { return g <= t.g_fp16 ? 4ll * g : 4ll * t.g_fp16 + (g - t.g_fp16); };
+    auto cost_before = [&](int g) {
+      return g <= t.g_fp16 ? (long long)kCostFp16 * g : (long long)kCostFp16 * t.g_fp16 + (long long)kCostQuant * (g - t.g_fp16);
+    };
     const long long total = cost_before(G);
     p.g_bounds[0] = 0;
     for (int sp = 1; sp < S; ++sp) {
