@@ -296,9 +296,20 @@ def profile_shape(args):
     us = ts[len(ts) // 2]
     nb = gemm_bytes(d_in, d_out, M, qbits, ks)
     assert ctx.last_status() == 0
-    print(json.dumps({"shape": f"{d_in}x{d_out}", "M": M, "bits": bits, "copies": copies, "us": round(us, 3),
-                      "us_min": round(ts[0], 3), "gbs": round(nb / us / 1e3, 1),
-                      "tflops": round(2.0 * M * d_in * d_out / us / 1e6, 1)}))
+    line = {"shape": f"{d_in}x{d_out}", "M": M, "bits": bits, "copies": copies, "us": round(us, 3),
+            "us_min": round(ts[0], 3), "gbs": round(nb / us / 1e3, 1),
+            "frac_of_measured": round(nb / us / 1e3 / load_peaks()["hbm_gbs"], 4),
+            "tflops": round(2.0 * M * d_in * d_out / us / 1e6, 1)}
+    if args.with_cublas:                                   # an fp16 GEMM of the same shape, same replay harness
+        for w in ws:
+            w.free()
+        fcopies = max(2, int(np.ceil(2 * 126e6 / (d_in * d_out * 2))))
+        Wf = [(torch.randn((d_in, d_out), device="cuda", generator=g) * 0.02).half() for _ in range(fcopies)]
+        gf = capture(lambda: [torch.matmul(x, w, out=y) for w in Wf])
+        tf = sorted(time_graphs([gf], 1, 1) * 1e3 / fcopies for _ in range(args.steps))
+        line["cublas_fp16_us"] = round(tf[len(tf) // 2], 3)
+        line["speedup_vs_cublas_fp16"] = round(tf[len(tf) // 2] / us, 3)
+    print(json.dumps(line))
 
 
 def calib_cov_throughput(ctx, peaks, n_tokens=16384, d=5120, reps=5):
@@ -482,6 +493,7 @@ def main():
     ap.add_argument("--profile-cov", type=int, nargs=2, metavar=("TOKENS", "D"),
                     help="time rosaq_calib_cov alone on TOKENS x D fp16 activations and exit")
     ap.add_argument("--copies", type=int, default=0, help="--profile-shape: distinct weight copies (default: 2 x L2)")
+    ap.add_argument("--with-cublas", action="store_true", help="--profile-shape: also time a cuBLAS FP16 GEMM of the shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.profile_shape:

@@ -145,17 +145,6 @@ __device__ __forceinline__ void tc_mma8_ts(uint32_t d_tmem, uint32_t a_tmem, uin
       "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// the two MMAs of a 32-channel slice of an fp16 group
-__device__ __forceinline__ void tc_mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                           uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
-      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %3, q;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // ---- CTA pairs (cta_group::2): two CTAs of a cluster, ranks 2j and 2j + 1, drive one MMA stream
 template <uint32_t kCols>
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t holder_smem) {
@@ -228,11 +217,6 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
 }
 __device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ uint32_t cluster_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
 __device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
@@ -441,7 +425,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
   const uint32_t misc = bar_d_full + 8;                        // [0] TMEM base, [1] abort flag
   uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t *misc_ptr = reinterpret_cast<volatile uint32_t *>(gen + (misc - base));
-  const uint32_t p_buf = base;                                 // fp32 partial tile, aliases the rings afterwards
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int prob = 0;
