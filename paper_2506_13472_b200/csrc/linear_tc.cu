@@ -98,11 +98,13 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+// 3-D view {64 channels, tokens, 64-channel block} of the activations: one instruction fetches both
+// 64-channel halves of a group (issuing a TMA costs the single producer lane a few hundred cycles)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int tok, int blk) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::
           "r"(dst),
-      "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      "l"(map), "r"(bar), "r"(0), "r"(tok), "r"(blk)
       : "memory");
 }
 // The column count is an immediate on purpose: with a register operand the tools cannot see how much
@@ -523,8 +525,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
           tma_load_2d_pair(x_ring + slot * x_slot_bytes + MTL * 128, &xmap, lb, k0 + 64, mrow);
         } else {
           mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
-          tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, m0);
-          tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, m0);
+          tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, m0, k0 >> 6);
         }
       }
       // (in a pair the leader's barriers count the loads of both CTAs, and the peer stays until the
@@ -880,8 +881,7 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         if (!ab.wait(bar_empty + 8 * slot, rs.lap ^ 1u)) break;
         const int k0 = (g_block0 + g) * kGroup;
         mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
-        tma_load_2d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, k0, 0);
-        tma_load_2d(x_ring + slot * x_slot_bytes + MT * 128, &xmap, bar_x_full + 8 * slot, k0 + 64, 0);
+        tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, 0, k0 >> 6);
         if (++g == p.G && j + 1 < n_units) {
           g = 0;
           g_block0 = block0(++tile);
@@ -1102,6 +1102,18 @@ size_t smem_bytes(int MT, int NW, int NA) {
 }
 
 
+// {64 channels, tokens, 64-channel block} view of the row-major activations, box = one group (two blocks)
+// of MT tokens; rows past M are zero-filled by the copy
+bool encode_x_map3(EncodeTiledFn encode, CUtensorMap *map, const __half *x, int M, long long ldx, int d_in, int MT) {
+  const cuuint64_t dims[3] = {64, (cuuint64_t)M, (cuuint64_t)(d_in / 64)};
+  const cuuint64_t strides[2] = {(cuuint64_t)ldx * sizeof(__half), 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)MT, 2};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half *>(x), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 size_t sk_smem_bytes(int MT, int NW) {
   size_t b = 1024 + (size_t)kSkStages * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NW + 4 * kSkStages) + 16;
   return b < 80 * 1024 ? 80 * 1024 : b;
@@ -1150,16 +1162,7 @@ static int launch_linear_sk(const rosaq_ctx *ctx, const __half *x, long long ldx
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return ROSAQ_ERR_CUDA;
   CUtensorMap xmap;
-  {
-    const cuuint64_t dims[2] = {(cuuint64_t)t.d_in, (cuuint64_t)q.M};
-    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
-    const cuuint32_t box[2] = {64, (cuuint32_t)q.MT};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(x), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return ROSAQ_ERR_CUDA;
-  }
+  if (!encode_x_map3(encode, &xmap, x, q.M, ldx, t.d_in, q.MT)) return ROSAQ_ERR_CUDA;
   const size_t smem = sk_smem_bytes(q.MT, q.NW);
   const bool int3 = t.g_quant > 0 && t.bits == 3;
   auto kern = int3 ? linear_sk_kernel<3> : linear_sk_kernel<4>;
@@ -1316,7 +1319,9 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   }
 
   CUtensorMap xmap;
-  {
+  if (!pair) {
+    if (!encode_x_map3(encode, &xmap, x, M, ldx, t.d_in, p.MT)) return ROSAQ_ERR_CUDA;
+  } else {
     const cuuint64_t dims[2] = {(cuuint64_t)t.d_in, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(__half)};
     const cuuint32_t box[2] = {64, (cuuint32_t)MTL};
