@@ -111,3 +111,61 @@ def test_headwise_full_size_o_proj(ctx):
     assert ctx.last_status() == rb.ROSAQ_OK
     y_ref = orc.forward(x, qd, Rb16, perm)
     assert H.rel_fro(y[:, cols], y_ref) <= H.REL_TOL_Y
+
+
+def test_layer_chain_replayed_from_a_graph_gives_the_bits_of_separate_calls(ctx):
+    """rotate -> gate + up (one launch; at this size the equal-share kernel with its workspace exchange) ->
+    down, as the benchmark chains them: captured in a CUDA graph, so that consecutive kernels overlap through
+    programmatic dependent launch, and replayed back to back.  Every replay must give the bits of the same
+    three calls issued one by one with a synchronisation after each (random packed weights: only the
+    chaining is under test here, the values are covered above)."""
+    d, f, M = 4096, 11008, 64
+    g = torch.Generator(device="cuda").manual_seed(5)
+
+    def packed(d_in, d_out):
+        nq = d_in - 128
+        qw = torch.randint(-2 ** 31, 2 ** 31 - 1, (nq // 8, d_out), dtype=torch.int64, device="cuda", generator=g).to(torch.int32)
+        sc = (torch.rand((nq // 128, d_out), device="cuda", generator=g) * 0.01 + 0.001).half()
+        zr = torch.randint(0, 16, (nq // 128, d_out), device="cuda", generator=g).half()
+        sal = (torch.randn((128, d_out), device="cuda", generator=g) * 0.02).half()
+        return ctx.weight_import(d_in, d_out, 4, 128, 128, qw, sc, zr, sal)
+
+    wg, wu, wd = packed(d, f), packed(d, f), packed(f, d)
+    rot = ctx.rotation_create((torch.randn((d, d), device="cuda", generator=g) / d ** 0.5).half())
+    x = torch.randn((M, d), device="cuda", generator=g).half()
+    xr = torch.empty((M, d), dtype=torch.float16, device="cuda")
+    gate, up = (torch.empty((M, f), dtype=torch.float16, device="cuda") for _ in range(2))
+    down = torch.empty((M, d), dtype=torch.float16, device="cuda")
+
+    def chain(sync):
+        ctx.rotate(x, rot, out=xr)
+        sync()
+        ctx.linear_multi(xr, [wg, wu], None, outs=[gate, up])
+        sync()
+        ctx.linear(gate, wd, None, out=down)
+        sync()
+
+    chain(torch.cuda.synchronize)
+    assert ctx.last_status() == rb.ROSAQ_OK
+    want = [t.clone() for t in (xr, gate, up, down)]
+    assert all(bool(torch.isfinite(t).all()) for t in want)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        chain(lambda: None)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        chain(lambda: None)
+    for rounds in (1, 6):
+        for t in (xr, gate, up, down):
+            t.zero_()
+        for _ in range(rounds):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.last_status() == rb.ROSAQ_OK
+        for got, ref in zip((xr, gate, up, down), want):
+            assert torch.equal(got.view(torch.int16), ref.view(torch.int16))
+    for h in (wg, wu, wd, rot):
+        h.free()
