@@ -104,6 +104,15 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
  * Returns the previous value. */
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl);
 
+/* Test hook, host only (no GPU, no context): the cut that implementation 0 uses when it gives every CTA an
+ * equal share of a launch.  The launch has n_tiles column tiles of `groups` 128-channel groups each, the
+ * first g_fp16 of every tile fp16, the others quantized; the tile-major (tile, group) list is cut into
+ * n_ctas contiguous ranges of equal cost.  Writes n_ctas + 1 ascending positions to bounds (HOST memory;
+ * range i is [bounds[i], bounds[i + 1])).  Returns ROSAQ_OK, ROSAQ_ERR_INVALID_ARG (a non-positive size,
+ * g_fp16 > groups, NULL), or ROSAQ_ERR_UNSUPPORTED_SHAPE when the cut is not usable -- a range would be
+ * empty or touch more than two tiles -- in which case rosaq_linear splits K across clusters instead. */
+int rosaq_plan_equal_shares(int n_tiles, int groups, int g_fp16, int n_ctas, int32_t *bounds);
+
 /* ---- calibration: Eq. 4, left-hand side ---------------------------------------- */
 
 /*

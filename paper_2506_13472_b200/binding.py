@@ -22,6 +22,7 @@ EXPORTS = [
     "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_weight_export",
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
     "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_multi", "rosaq_linear_static",
+    "rosaq_plan_equal_shares",
 ]
 
 
@@ -72,6 +73,7 @@ def lib():
         L.rosaq_linear_static.argtypes = L.rosaq_linear.argtypes
         L.rosaq_linear_multi.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rosaq_plan_equal_shares.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32)]
         _lib = L
     return _lib
 
@@ -111,6 +113,13 @@ def _rot_struct(q, perm):
     if perm is not None:
         assert perm.is_cuda and perm.dtype == torch.int32 and perm.is_contiguous() and perm.numel() == nb * dh
     return _Rot(nb * dh, nb, q.data_ptr(), _dt(q), None if perm is None else perm.data_ptr())
+
+
+def plan_equal_shares(n_tiles, groups, g_fp16, n_ctas):
+    """rosaq_plan_equal_shares: the n_ctas + 1 bounds of the equal-share cut (host only), or RosaqError."""
+    out = (C.c_int32 * (max(n_ctas, 0) + 1))()
+    _check(lib().rosaq_plan_equal_shares(n_tiles, groups, g_fp16, n_ctas, out), "rosaq_plan_equal_shares")
+    return list(out)
 
 
 class Context:

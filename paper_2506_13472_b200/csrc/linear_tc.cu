@@ -1119,7 +1119,8 @@ size_t sk_smem_bytes(int MT, int NW) {
   return b < 80 * 1024 ? 80 * 1024 : b;
 }
 
-// Cuts the tile-major (tile, group) list into P ranges of equal cost, every cut on a group boundary.  False when a range would be empty or touch more than two tiles.
+// Cuts the tile-major (tile, group) list into P ranges of equal cost, every cut on a group boundary.
+// False when a range would be empty or touch more than two tiles.
 bool sk_bounds(int T, int G, int g_fp16, int P, int *bounds) {
   const long long FW = kCostFp16, QW = kCostQuant;
   const long long C = FW * g_fp16 + QW * (G - g_fp16), N = C * T;
@@ -1383,3 +1384,11 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
 }
 
 }  // namespace rosaq
+
+extern "C" int rosaq_plan_equal_shares(int n_tiles, int groups, int g_fp16, int n_ctas, int32_t *bounds) {
+  if (n_tiles <= 0 || groups <= 0 || g_fp16 < 0 || g_fp16 > groups || n_ctas <= 0 || !bounds) return ROSAQ_ERR_INVALID_ARG;
+  if ((long long)n_tiles * groups > 0x7fffffffll) return ROSAQ_ERR_INVALID_ARG;
+  static_assert(sizeof(int) == sizeof(int32_t), "bounds are written as int");
+  return rosaq::sk_bounds(n_tiles, groups, g_fp16, n_ctas, reinterpret_cast<int *>(bounds)) ? ROSAQ_OK
+                                                                                           : ROSAQ_ERR_UNSUPPORTED_SHAPE;
+}
