@@ -453,7 +453,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
     }
     for (int i = 0; i < p.NA; ++i) {
       mbar_init(bar_x_full + 8 * i, 1);
-      mbar_init(bar_a_full + 8 * i, n_arrive);
+      mbar_init(bar_a_full + 8 * i, kPair ? n_arrive : n_arrive + 1);   // + the activation copy (single-CTA mode)
       mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_d_full, 1);
@@ -524,17 +524,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
           tma_load_2d_pair(x_ring + slot * x_slot_bytes, &xmap, lb, k0, mrow);
           tma_load_2d_pair(x_ring + slot * x_slot_bytes + MTL * 128, &xmap, lb, k0 + 64, mrow);
         } else {
-          mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
-          tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, m0, k0 >> 6);
+          // the copy completes on the stage's operand barrier: the MMA thread then polls one barrier per group
+          mbar_arrive_expect_tx(bar_a_full + 8 * slot, x_slot_bytes);
+          tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_a_full + 8 * slot, m0, k0 >> 6);
         }
       }
       // (in a pair the leader's barriers count the loads of both CTAs, and the peer stays until the
       // cluster barrier at the end of the kernel, which the leader reaches after this drain)
       if (ab.set() && is_lead) {
+        const uint32_t bar_copy = kPair ? bar_x_full : bar_a_full;
         for (int back = 1; back <= p.NA && back <= gc; ++back) {
           const int u = gc - back;
           for (int it = 0; it < kDrainPolls; ++it)
-            if (ab.poll(bar_x_full + 8 * (u % p.NA), (u / p.NA) & 1)) break;
+            if (ab.poll(bar_copy + 8 * (u % p.NA), (u / p.NA) & 1)) break;
         }
       }
     }
@@ -550,7 +552,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap xmap, const TcParams p) {
       uint32_t accumulate = 0;
       for (int g = g_begin; g < g_end; ++g, rs.advance(p.NA)) {
         const int st = rs.idx;
-        if (!ab.wait(bar_x_full + 8 * st, rs.lap) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
+        if ((kPair && !ab.wait(bar_x_full + 8 * st, rs.lap)) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
         tc_fence_after();
         const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
         if (kPair) {
@@ -810,7 +812,7 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
     }
     for (int i = 0; i < kSkStages; ++i) {
       mbar_init(bar_x_full + 8 * i, 1);
-      mbar_init(bar_a_full + 8 * i, kTeamThreads);
+      mbar_init(bar_a_full + 8 * i, kTeamThreads + 1);         // + the activation copy
       mbar_init(bar_empty + 8 * i, 1);
       mbar_init(bar_d_full + 8 * i, 1);
     }
@@ -880,8 +882,8 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         const int slot = rs.idx;
         if (!ab.wait(bar_empty + 8 * slot, rs.lap ^ 1u)) break;
         const int k0 = (g_block0 + g) * kGroup;
-        mbar_arrive_expect_tx(bar_x_full + 8 * slot, x_slot_bytes);
-        tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_x_full + 8 * slot, 0, k0 >> 6);
+        mbar_arrive_expect_tx(bar_a_full + 8 * slot, x_slot_bytes);
+        tma_load_3d(x_ring + slot * x_slot_bytes, &xmap, bar_a_full + 8 * slot, 0, k0 >> 6);
         if (++g == p.G && j + 1 < n_units) {
           g = 0;
           g_block0 = block0(++tile);
@@ -891,7 +893,7 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         for (int back = 1; back <= kSkStages && back <= gc; ++back) {
           const int u = gc - back;
           for (int it = 0; it < kDrainPolls; ++it)
-            if (mbar_try_wait(bar_x_full + 8 * (u % kSkStages), (u / kSkStages) & 1)) break;
+            if (mbar_try_wait(bar_a_full + 8 * (u % kSkStages), (u / kSkStages) & 1)) break;
         }
       }
     }
@@ -906,7 +908,7 @@ linear_sk_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
       int g = g0, seg = 0, committed = 0;
       for (int j = 0; j < n_units; ++j, rs.advance(kSkStages)) {
         const int st = rs.idx;
-        if (!ab.wait(bar_x_full + 8 * st, rs.lap) || !ab.wait(bar_a_full + 8 * st, rs.lap)) break;
+        if (!ab.wait(bar_a_full + 8 * st, rs.lap)) break;
         tc_fence_after();
         const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
         tc_mma8_ts(tmem + seg * kSkTokens, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
