@@ -1260,8 +1260,8 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   for (int i = 0; i < n && pair; ++i) pair = ts[i]->n_tiles % 2 == 0;
   // stream-K variant: token tile of at most 64 tokens, one token tile, and so many column tiles that a tile
   // is shared by two or three CTAs at most (its finisher reads the others' partial tiles one after the
-  // other; measured at 64 tokens: 4096 -> 22016, 172 tiles, 24.1 us against 28.4 with cluster splits;
-  // with 96 tiles equal, with 86 tiles 1.7 us slower)
+  // other; measured at 64 tokens: 4096 -> 22016, 172 tiles, 23.4 us against 28.4 with cluster splits;
+  // with 96 tiles 0.7 us slower, with 86 tiles 2.2 us slower)
   if (ctx->impl == 0 && !pair && m_tiles == 1 && p.MT <= kSkTokens && ctx->sk_partials && tc_overrides().sk > 0) {
     const int P = ctx->sk_ctas < 2 * ctx->sm_count ? ctx->sk_ctas : 2 * ctx->sm_count;
     if (n_tiles_all <= P && n_tiles_all <= kSkCounterInts && (long long)n_tiles_all * tc_overrides().sk >= P) {
