@@ -200,8 +200,11 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
 
 /*
  * Several linears that read the same activation (q/k/v, or gate/up: they share one rotation, Section 3.1)
- * in one launch:  y[i] = (x . R) . W^[i]  for i < n, 1 <= n <= 4, each with the result bits rosaq_linear
- * would give.  All w[i] must have the same d_in, bits and k_salient; d_out may differ.  w, y and ldy are
+ * in one launch:  y[i] = (x . R) . W^[i]  for i < n, 1 <= n <= 4.  Each y[i] is the sum rosaq_linear would
+ * compute; how K is split among CTAs depends on the number of column tiles in a launch, so the two agree
+ * to fp32 summation order -- bit for bit where the splits coincide (small operands), within a few 1e-5
+ * relative otherwise.  Repeated launches of the same call always give the same bits.
+ * All w[i] must have the same d_in, bits and k_salient; d_out may differ.  w, y and ldy are
  * HOST arrays of n entries (device pointers inside); they are read before the call returns.
  * r as in rosaq_linear (the rotation runs once).  Errors as rosaq_linear.
  */
