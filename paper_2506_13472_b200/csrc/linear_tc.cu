@@ -22,7 +22,7 @@
 // status word, stops issuing work, still joins the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
 
-#include "rosaq_internal.cuh"
+#include "linear_common.cuh"
 
 namespace rosaq {
 
@@ -30,10 +30,7 @@ namespace {
 
 constexpr int kThreads = 352;
 constexpr int kDequantThreads = 256;
-constexpr int kTeamThreads = 128;                          // one dequantisation team: a warp per TMEM lane quadrant
 constexpr int kFirstDequantWarp = 3;
-constexpr int kWSlotBytes = kInt4CodeBytes + kScaleBytes;  // 8704: one quantized tile or a quarter fp16 tile
-constexpr int kFp16SubBytes = kFp16TileBytes / 4;          // 32 input channels of an fp16 tile
 constexpr int kTmemCols = 256;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxProblems = 4;   // weights sharing one activation in a launch (q/k/v, gate/up)
@@ -42,10 +39,6 @@ constexpr int kMaxSplits = 8;
 // but up to 64 tokens a CTA is paced by its eight MMAs and its handshakes per group, not by bytes
 // (measured: weights 4 : 1 lose 2-5 % against 1.5 : 1 on the 7B shapes).
 constexpr int kCostFp16 = 3, kCostQuant = 2;
-// polls (about a microsecond each) granted to work already in flight when a CTA gives up: unlike the
-// waits of the pipeline this bound does not follow the context's wait limit, so that a shortened limit
-// can never let a CTA retire under its own copies or MMAs
-constexpr int kDrainPolls = 1 << 16;
 
 struct TcParams {
   // up to kMaxProblems weights of identical geometry (d_in, bits, salient groups) that multiply the same
@@ -67,342 +60,6 @@ struct TcParams {
   int NW, NA;                // ring depths: packed-weight slots, stages (TMEM A buffer + activation slot)
 };
 
-// ---------------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// One poll of a barrier phase.  The suspend-time hint lets the hardware park the thread (up to about
-// a microsecond, woken as soon as the phase completes) instead of returning at once: warps that wait
-// then stop competing for issue slots with the warps that work.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(1000u)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-// 3-D view {64 channels, tokens, 64-channel block} of the activations: one instruction fetches both
-// 64-channel halves of a group (issuing a TMA costs the single producer lane a few hundred cycles)
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int tok, int blk) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::
-          "r"(dst),
-      "l"(map), "r"(bar), "r"(0), "r"(tok), "r"(blk)
-      : "memory");
-}
-// The column count is an immediate on purpose: with a register operand the tools cannot see how much
-// tensor memory a CTA takes and assume all 512 columns, which limits the kernel to one CTA per SM.
-template <uint32_t kCols>
-__device__ __forceinline__ void tmem_alloc(uint32_t holder_smem) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "n"(kCols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-template <uint32_t kCols>
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "n"(kCols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]; fp16 inputs, fp32 accumulate.  The MMAs of one unit are
-// emitted as one block of back-to-back instructions sharing their predicates: issued one by one from
-// separate statements they cost the issuing thread about 100 cycles each, in a block about 45.
-// A advances by 8 TMEM columns (16 input channels) per MMA; B by 32 bytes inside a 64-channel
-// swizzle row (descriptor address field + 2), b_hi is the descriptor of the second 64-channel half.
-__device__ __forceinline__ void tc_mma8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_lo, uint64_t b_hi,
-                                           uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, p;\n\t"
-      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 16;\n\tadd.u64 t, %2, 4;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 24;\n\tadd.u64 t, %2, 6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 32;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], %3, %4, q;\n\t"
-      "add.u32 a, %1, 40;\n\tadd.u64 t, %3, 2;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 48;\n\tadd.u64 t, %3, 4;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 56;\n\tadd.u64 t, %3, 6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], t, %4, q;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// ---- CTA pairs (cta_group::2): two CTAs of a cluster, ranks 2j and 2j + 1, drive one MMA stream
-template <uint32_t kCols>
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t holder_smem) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "n"(kCols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-template <uint32_t kCols>
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "n"(kCols) : "memory");
-}
-// commit whose arrival is delivered to the barrier at the same offset in every CTA of `mask`
-__device__ __forceinline__ void tc_commit_mc(uint32_t bar, uint32_t mask) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-      "h"((unsigned short)mask)
-      : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// load whose bytes are counted on a barrier of the pair's leader (a shared::cluster address); no multicast
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t lead_bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
-          "r"(dst),
-      "l"(map), "r"(lead_bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(1000u)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void tc_mma8_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_lo, uint64_t b_hi,
-                                                uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 t;\n\t.reg .b32 a;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %4, p;\n\t"
-      "add.u32 a, %1, 8;\n\tadd.u64 t, %2, 2;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 16;\n\tadd.u64 t, %2, 4;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 24;\n\tadd.u64 t, %2, 6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 32;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], %3, %4, q;\n\t"
-      "add.u32 a, %1, 40;\n\tadd.u64 t, %3, 2;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 48;\n\tadd.u64 t, %3, 4;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t"
-      "add.u32 a, %1, 56;\n\tadd.u64 t, %3, 6;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [a], t, %4, q;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_lo), "l"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
-          taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
-}
-__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
-__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & mask) | orv
-  return r;
-}
-__device__ __forceinline__ uint32_t h2_sub_mul(uint32_t v, uint32_t sub, uint32_t mul) {
-  __half2 r = __hmul2(__hsub2(*reinterpret_cast<__half2 *>(&v), *reinterpret_cast<__half2 *>(&sub)),
-                      *reinterpret_cast<__half2 *>(&mul));
-  return *reinterpret_cast<uint32_t *>(&r);
-}
-
-// K-major, 128-byte-swizzled shared-memory operand: 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_b_desc(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr >> 4) & 0x3fff) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-
-// ---------------------------------------------------------------------------------- dequantisation
-// (code - zero) * scale in fp16, exact subtraction then one rounding: codes are spliced into the
-// mantissa of a power-of-two constant (1024, 128, 64 or 16 depending on the bit position), which
-// turns them into fp16 integers without a conversion instruction.
-struct ScaleZero {
-  uint32_t s2, z1024, z128, z64, z16;
-  __device__ __forceinline__ explicit ScaleZero(uint32_t sz) {
-    const uint32_t s = sz & 0xffffu, z = sz >> 16;
-    s2 = s | (s << 16);
-    const uint32_t zz = z | (z << 16);
-    auto add = [&](uint32_t c) {
-      __half2 r = __hadd2(*reinterpret_cast<const __half2 *>(&zz), *reinterpret_cast<const __half2 *>(&c));
-      return *reinterpret_cast<uint32_t *>(&r);
-    };
-    z1024 = add(0x64006400u);
-    z128 = add(0x58005800u);
-    z64 = add(0x54005400u);
-    z16 = add(0x4C004C00u);
-  }
-};
-
-// one word = 8 INT4 codes -> 4 fp16 pairs (k, k+1), (k+2, k+3), (k+4, k+5), (k+6, k+7)
-__device__ __forceinline__ void dequant_int4_word(uint32_t q, const ScaleZero &c, uint32_t *out) {
-  const uint32_t q8 = q >> 8;
-  out[0] = h2_sub_mul(lop_and_or(q, 0x000f000fu, 0x64006400u), c.z1024, c.s2);
-  out[1] = h2_sub_mul(lop_and_or(q, 0x00f000f0u, 0x54005400u), c.z64, c.s2);
-  out[2] = h2_sub_mul(lop_and_or(q8, 0x000f000fu, 0x64006400u), c.z1024, c.s2);
-  out[3] = h2_sub_mul(lop_and_or(q8, 0x00f000f0u, 0x54005400u), c.z64, c.s2);
-}
-
-// three words = 32 INT3 codes -> 16 fp16 pairs
-__device__ __forceinline__ void dequant_int3_set(uint32_t a, uint32_t b, uint32_t cc, const ScaleZero &c,
-                                                 uint32_t *out) {
-  const uint32_t w[3] = {a, b, cc};
-#pragma unroll
-  for (int i = 0; i < 3; ++i) {
-    const uint32_t q = w[i], q9 = q >> 9;
-    out[5 * i + 0] = h2_sub_mul(lop_and_or(q, 0x00070007u, 0x64006400u), c.z1024, c.s2);
-    out[5 * i + 1] = h2_sub_mul(lop_and_or(q, 0x00380038u, 0x58005800u), c.z128, c.s2);
-    out[5 * i + 2] = h2_sub_mul(lop_and_or(q, 0x01c001c0u, 0x4C004C00u), c.z16, c.s2);
-    out[5 * i + 3] = h2_sub_mul(lop_and_or(q9, 0x00070007u, 0x64006400u), c.z1024, c.s2);
-    out[5 * i + 4] = h2_sub_mul(lop_and_or(q9, 0x00380038u, 0x58005800u), c.z128, c.s2);
-  }
-  const uint32_t tail = ((a >> 15) & 0x00010001u) | ((b >> 14) & 0x00020002u) | ((cc >> 13) & 0x00040004u);
-  out[15] = h2_sub_mul(tail | 0x64006400u, c.z1024, c.s2);
-}
-
-// One unit of the weight ring (a quantized group, or 32 input channels of an fp16 group) of output
-// column n: shared memory -> registers -> the TMEM operand buffer at a_addr.  The slot is released
-// only after instructions that depend on every loaded word have been issued: an arrive placed right
-// behind the loads can be performed while they are still queued (seen when the other CTA of the SM kept
-// the load/store unit busy with global stores), and the producer then refills the slot under them.
-template <int kBits>
-__device__ __forceinline__ void dequant_unit(bool f16, uint32_t slot_base, int n, uint32_t a_addr, int sub,
-                                             uint32_t bar_release) {
-  const uint32_t ws = slot_base + n * 16;
-  if (f16) {
-    // a quarter of an fp16 group: 32 input channels = 16 TMEM columns
-    uint32_t r[16];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4 *>(&r[4 * j]) = lds128(ws + j * (kTileN * 16));
-    tmem_st16(a_addr + 16 * sub, r);
-    mbar_arrive(bar_release);
-  } else if (kBits == 4) {
-    const ScaleZero c(lds32(slot_base + kInt4CodeBytes + n * 4));
-    uint4 q[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) q[j] = lds128(ws + j * (kTileN * 16));
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t r[16];
-      dequant_int4_word(q[j].x, c, &r[0]);
-      dequant_int4_word(q[j].y, c, &r[4]);
-      dequant_int4_word(q[j].z, c, &r[8]);
-      dequant_int4_word(q[j].w, c, &r[12]);
-      tmem_st16(a_addr + 16 * j, r);
-    }
-    mbar_arrive(bar_release);
-  } else {
-    const ScaleZero c(lds32(slot_base + kInt3CodeBytes + n * 4));
-    // the column's 12 words: 4 sets of 3 words = 32 codes = 16 TMEM columns each
-    uint32_t w12[12];
-#pragma unroll
-    for (int j = 0; j < 3; ++j) *reinterpret_cast<uint4 *>(&w12[4 * j]) = lds128(ws + j * (kTileN * 16));
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t r[16];
-      dequant_int3_set(w12[3 * j], w12[3 * j + 1], w12[3 * j + 2], c, r);
-      tmem_st16(a_addr + 16 * j, r);
-    }
-    mbar_arrive(bar_release);
-  }
-}
-
-// ---------------------------------------------------------------------------------- the kernel
-struct Abort {
-  volatile int *flag;     // shared
-  int *status;            // global
-  long long limit;
-  bool cluster_scope;     // barriers also receive arrivals from the peer CTA of a pair
-  __device__ __forceinline__ bool set() const { return *flag != 0; }
-  __device__ __forceinline__ void raise() const {
-    *flag = 1;
-    atomicExch(status, (int)ROSAQ_ERR_TIMEOUT);
-  }
-  // false when the wait gave up (or somebody else already did)
-  __device__ __forceinline__ bool poll(uint32_t bar, uint32_t parity) const {
-    return cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
-  }
-  // barriers that only this CTA's threads and copies feed: CTA scope whatever the mode
-  __device__ __forceinline__ bool wait_local(uint32_t bar, uint32_t parity) const {
-    if (mbar_try_wait(bar, parity)) return true;
-    for (long long it = 0; it < limit; ++it) {
-      if (mbar_try_wait(bar, parity)) return true;
-      if ((it & 63) == 63 && set()) return false;
-    }
-    raise();
-    return false;
-  }
-  // one cluster-scope poll per warp instead of thirty-two, verdict broadcast (also the warp-level sync)
-  __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity) const {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = wait(bar, parity) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
-  }
-  __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
-    if (poll(bar, parity)) return true;
-    for (long long it = 0; it < limit; ++it) {
-      if (poll(bar, parity)) return true;
-      if ((it & 63) == 63 && set()) return false;
-    }
-    raise();
-    return false;
-  }
-};
-
-// Position in a ring of n slots plus the parity of the current lap, advanced without division
-// (the role warps run on a single lane: an integer division there costs hundreds of cycles).
-struct Ring {
-  int idx;
-  uint32_t lap;
-  __device__ __forceinline__ void advance(int n) {
-    if (++idx == n) {
-      idx = 0;
-      lap ^= 1u;
-    }
-  }
-};
 
 // kPair: two CTAs with adjacent column tiles (cluster ranks 2j, 2j + 1; blockIdx.x even / odd) run as a
 // cta_group::2 pair.  Each dequantises its own 128 columns into its own tensor memory and loads half of

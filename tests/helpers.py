@@ -79,3 +79,54 @@ def cov_tolerance(Cref, n_tokens):
     dg = np.sqrt(np.clip(np.diagonal(Cref, axis1=-2, axis2=-1), 0, None))
     steps = max(4.0 * np.sqrt(n_tokens) + 8.0, 2.0 * (n_tokens / 16.0 + 8.0))
     return 2.0 ** -24 * steps * dg[..., :, None] * dg[..., None, :]
+
+
+def qd_from_export(exported, bits, k_salient, group=128):
+    """The oracle's weight dict built from a GPU export (numpy arrays, all columns): what
+    orc.forward needs to compute y_ref on exactly the weights the GPU holds."""
+    d_q = exported["scales"].shape[0] * group
+    codes = (orc.unpack(exported["qw"].view(np.uint32), d_q, bits) if d_q
+             else np.zeros((0, exported["salient"].shape[1]), np.uint8))
+    return dict(salient=exported["salient"], scales=exported["scales"], zeros=exported["zeros"], codes=codes,
+                bits=bits, group=group, k_salient=k_salient)
+
+
+def tile_columns(d_out, seed, key, tile=128):
+    """One seeded column out of every `tile`-column tile, plus the first and last column of the matrix
+    and both sides of the first tile edge."""
+    rng = synth.rng_for(seed, key, "tilecols")
+    cols = {0, d_out - 1, min(tile - 1, d_out - 1), min(tile, d_out - 1)}
+    for t0 in range(0, d_out, tile):
+        cols.add(int(t0 + rng.integers(0, min(tile, d_out - t0))))
+    return np.asarray(sorted(cols), dtype=np.int32)
+
+
+def assert_y_all_columns(y, x_in16, qd, tile=128, chunk=2048, where=""):
+    """y (fp16, every column) against the oracle's fp64 forward on the same activations and the same
+    dequantised weights:  the 2e-3 Frobenius bound on every `tile`-column tile (a bad tile cannot hide
+    in the norm of the whole matrix), and element by element
+        |y - y_ref| <= 2e-3 * (|x| . |W^|)_mn + ulp_fp16(y_ref)
+    (the products carry at most one fp16 rounding of W^ each, the sum is fp32, y is rounded once).
+    x_in16 is what the GEMM stage was fed (already rotated)."""
+    y = np.asarray(y)
+    M, d_out = y.shape
+    assert np.all(np.isfinite(y)), where
+    xa = np.abs(orc.f16_to_f64(np.ascontiguousarray(x_in16, np.float16)))
+    worst_tile, worst_elem = 0.0, 0.0
+    for c0 in range(0, d_out, chunk):
+        c1 = min(c0 + chunk, d_out)
+        sub = dict(qd, salient=qd["salient"][:, c0:c1], scales=qd["scales"][:, c0:c1], zeros=qd["zeros"][:, c0:c1],
+                   codes=qd["codes"][:, c0:c1])
+        y_ref = orc.forward(x_in16, sub)
+        mag = xa @ np.abs(orc.dequantize(sub))
+        got = y[:, c0:c1].astype(np.float64)
+        bound = REL_TOL_Y * mag + np.spacing(np.abs(y_ref).astype(np.float16)).astype(np.float64)
+        ratio = np.abs(got - y_ref) / np.maximum(bound, 1e-300)
+        worst_elem = max(worst_elem, float(ratio.max()))
+        bad = np.argwhere(ratio > 1.0)
+        assert bad.size == 0, f"{where}: element (token {bad[0][0]}, column {c0 + bad[0][1]}) off by {ratio.max():.2f} bounds"
+        for t0 in range(0, c1 - c0, tile):
+            e = rel_fro(got[:, t0:t0 + tile], y_ref[:, t0:t0 + tile])
+            worst_tile = max(worst_tile, e)
+            assert e <= REL_TOL_Y, f"{where}: columns {c0 + t0}..{c0 + t0 + tile - 1}: {e:.2e}"
+    return worst_tile, worst_elem

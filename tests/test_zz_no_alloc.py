@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import rosaq_oracle as orc
 from paper_2506_13472_b200 import binding as rb
 from paper_2506_13472_b200 import synth
 from tests import helpers as H
@@ -32,12 +33,14 @@ def test_static_variant_matches_rosaq_linear_on_two_calls_in_a_row():
     try:
         c = H.config_headwise()                     # block-diagonal R with a permutation, d_in = 512
         w = ctx.quantize(dev(c["W"]), dev(c["Rb32"]), dev(c["perm"]), bits=4, k_salient=128)
+        qd = H.oracle_quantized(c["W"], c["Rb32"], c["perm"], 4, 128)
         rot = ctx.rotation_create(dev(c["Rb16"]), dev(c["perm"]))
         law = synth.HeadwiseActivationLaw(c["heads"], c["head_dim"], 3, "hw")
         # first call: 37 tokens; second call: fewer tokens and other values, so stale rows of the
         # shared array from the first call would show up if they were read
         for M, tag in ((37, "static-a"), (5, "static-b")):
-            x = dev(law.sample(M, tag, np.float16))
+            x16 = law.sample(M, tag, np.float16)
+            x = dev(x16)
             want = ctx.linear(x, w, rot)
             got = torch.full((M, w.d_out), float("nan"), dtype=torch.float16, device="cuda")
             ctx.linear_static(x, w, rot, out=got)
@@ -46,6 +49,8 @@ def test_static_variant_matches_rosaq_linear_on_two_calls_in_a_row():
             assert np.all(np.isfinite(got))
             assert H.rel_fro(got, want) <= H.REL_TOL_Y
             assert np.array_equal(got.view(np.uint16), want.view(np.uint16))   # same kernels, same bits
+            # and on its own feet: the CPU oracle's fp64 forward on the same inputs
+            assert H.rel_fro(got, orc.forward(x16, qd, c["Rb16"], c["perm"])) <= H.REL_TOL_Y
         # r == NULL needs no scratch: plain GEMM stage on pre-rotated input
         xr = ctx.rotate(dev(law.sample(9, "static-c", np.float16)), rot)
         a = ctx.linear(xr, w, None).cpu().numpy()
