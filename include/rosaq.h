@@ -51,6 +51,7 @@ typedef enum { ROSAQ_F16 = 0, ROSAQ_F32 = 1 } rosaq_dtype;
 typedef struct rosaq_ctx rosaq_ctx;           /* per device: workspace + device status word */
 typedef struct rosaq_weight rosaq_weight;     /* one quantized linear in the kernels' tiled layout */
 typedef struct rosaq_rotation rosaq_rotation; /* one rotation R prepared for online use */
+typedef struct rosaq_plan rosaq_plan;         /* a list of rotations / linears that runs as one launch */
 
 /*
  * Description of a rotation R (Section 3.1, Eq. 4; head-wise: Section 3.1.1, Eq. 6).
@@ -210,6 +211,64 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
  */
 int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r, int n,
                        const rosaq_weight *const *w, void *const *y, const int64_t *ldy, void *stream);
+
+/*
+ * A list of operations that runs as ONE persistent launch (up to 64 tokens): every rotation x . R
+ * (Eq. 2; Eq. 6 for block-diagonal R) and every GEMM stage x' . W^ (Eq. 3) of, say, a decoder layer.
+ * All CTAs of the grid stream the operands of the whole list back to back; an operation whose input is
+ * another operation's output starts when that output is complete.
+ *   op.r / op.w  exactly one is non-NULL: the operation is y = x . R, or y = x . W^ (x already rotated)
+ *   op.x, ldx    DEVICE [M][ldx] fp16 input; ignored when x_from >= 0
+ *   op.x_from    -1, or the index (smaller than this operation's) of the operation whose y is this one's
+ *                input (a rotation feeding its linears); that y must have this operation's d_in columns
+ *   op.y, ldy    DEVICE [M][ldy] fp16 output; the first d_out columns of each row are written
+ * Operations without x_from are independent of each other and may run in any order or at the same time;
+ * the caller guarantees that no y overlaps any other operation's x or y.  All quantized weights of a list
+ * have the same bit width.  1 <= M <= 64 and 1 <= n_ops <= 12, otherwise ROSAQ_ERR_UNSUPPORTED_SHAPE.
+ * Each y is the sum rosaq_linear computes, added in an order that depends on how the list is divided
+ * among the CTAs: results agree with the separate calls to fp32 summation order (a few 1e-5 relative) and
+ * are the same bits on every run of the same plan.
+ * rosaq_plan_create reads `ops` (HOST array) before it returns, may allocate device memory and may
+ * synchronize the device; create the plans a CUDA graph will replay before capturing it.
+ * rosaq_plan_run launches on `stream` and allocates nothing; runs of plans of one context must not
+ * overlap on the GPU (they share the context's exchange workspace): keep them on one stream.
+ * The pointers inside ops, and the rotation and weight handles, must stay valid while the plan is used.
+ */
+typedef struct {
+  const void *x;
+  int64_t ldx;
+  int32_t x_from;
+  const rosaq_rotation *r;
+  const rosaq_weight *w;
+  void *y;
+  int64_t ldy;
+} rosaq_op;
+int rosaq_plan_create(rosaq_ctx *ctx, int M, int n_ops, const rosaq_op *ops, rosaq_plan **out);
+int rosaq_plan_run(rosaq_ctx *ctx, const rosaq_plan *plan, void *stream);
+int rosaq_plan_free(rosaq_plan *plan);
+
+/* Number of CTAs of the persistent launch on the context's device (two per SM), or a negative status. */
+int rosaq_plan_ctas(rosaq_ctx *ctx);
+
+/*
+ * Test hook, host only (no GPU, no context): how a list of operations is divided among n_ctas CTAs.
+ * Operation i has n_tiles[i] column tiles of groups[i] 128-channel groups, the first g_fp16[i] of each
+ * tile fp16; x_from[i] as in rosaq_op; copies[i] >= 1 (NULL: all 1) computes every tile of the operation that
+ * many times, each copy writing an equal share of the token rows (what the library does, four-fold, for
+ * block-diagonal rotations with a column permutation, whose output is a scatter bound by the store rate
+ * of one SM).  An operation runs in the phase after the one it reads from; inside
+ * a phase the (operation, tile, group) list is cut into n_ctas contiguous ranges of equal cost, and a
+ * range is a sequence of pieces (the groups of one tile).  Writes piece_begin[0..n_ctas] (CTA c owns pieces
+ * piece_begin[c] .. piece_begin[c + 1] - 1, in the order it processes them) and, for the first max_pieces
+ * pieces, twelve int32 each: operation, tile, first group, end group, holders of the tile (copy), this
+ * piece's position among them (ascending K), first partial-tile slot, arrival counter, closer index (-1: the
+ * piece only contributes its partial tile; k >= 0: its CTA adds the partial tiles of token rows k,
+ * k + closers, ...), closers, and the token rows [begin, end) out of 64 that the tile (copy) writes.
+ * All arrays HOST.  Returns the total number of pieces, or a negative status.
+ */
+int rosaq_plan_schedule(int n_ops, const int32_t *n_tiles, const int32_t *groups, const int32_t *g_fp16,
+                        const int32_t *x_from, const int32_t *copies, int n_ctas, int32_t *piece_begin,
+                        int32_t *pieces, int max_pieces);
 
 /*
  * Same result as rosaq_linear, for callers that cannot allocate device memory.  (The paper has

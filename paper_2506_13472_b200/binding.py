@@ -22,7 +22,8 @@ EXPORTS = [
     "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_weight_export",
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
     "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_multi", "rosaq_linear_static",
-    "rosaq_plan_equal_shares",
+    "rosaq_plan_equal_shares", "rosaq_plan_create", "rosaq_plan_run", "rosaq_plan_free", "rosaq_plan_ctas",
+    "rosaq_plan_schedule",
 ]
 
 
@@ -35,6 +36,11 @@ class RosaqError(RuntimeError):
 class _Rot(C.Structure):
     _fields_ = [("d", C.c_int32), ("n_blocks", C.c_int32), ("q", C.c_void_p), ("q_dtype", C.c_int32),
                 ("perm", C.c_void_p)]
+
+
+class _Op(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("ldx", C.c_int64), ("x_from", C.c_int32), ("r", C.c_void_p), ("w", C.c_void_p),
+                ("y", C.c_void_p), ("ldy", C.c_int64)]
 
 
 _lib = None
@@ -74,6 +80,12 @@ def lib():
         L.rosaq_linear_multi.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
         L.rosaq_plan_equal_shares.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32)]
+        L.rosaq_plan_create.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(_Op), C.POINTER(C.c_void_p)]
+        L.rosaq_plan_run.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rosaq_plan_free.argtypes = [C.c_void_p]
+        L.rosaq_plan_ctas.argtypes = [C.c_void_p]
+        L.rosaq_plan_schedule.argtypes = [C.c_int] + [C.POINTER(C.c_int32)] * 5 + [C.c_int, C.POINTER(C.c_int32),
+                                                                                  C.POINTER(C.c_int32), C.c_int]
         _lib = L
     return _lib
 
@@ -120,6 +132,26 @@ def plan_equal_shares(n_tiles, groups, g_fp16, n_ctas):
     out = (C.c_int32 * (max(n_ctas, 0) + 1))()
     _check(lib().rosaq_plan_equal_shares(n_tiles, groups, g_fp16, n_ctas, out), "rosaq_plan_equal_shares")
     return list(out)
+
+
+PIECE_FIELDS = ("op", "tile", "g_begin", "g_end", "holders", "holder_idx", "slot0", "counter", "closer_idx", "closers",
+                "tok_begin", "tok_end")
+
+
+def plan_schedule(n_tiles, groups, g_fp16, x_from, n_ctas, copies=None):
+    """rosaq_plan_schedule (host only): (piece_begin, pieces) with pieces a list of dicts keyed by PIECE_FIELDS."""
+    n = len(n_tiles)
+    arr = lambda v: (C.c_int32 * n)(*[int(a) for a in v])
+    begin = (C.c_int32 * (n_ctas + 1))()
+    args = (n, arr(n_tiles), arr(groups), arr(g_fp16), arr(x_from), None if copies is None else arr(copies), n_ctas, begin)
+    total = lib().rosaq_plan_schedule(*args, None, 0)
+    if total < 0:
+        raise RosaqError(total, "rosaq_plan_schedule")
+    raw = (C.c_int32 * (12 * max(total, 1)))()
+    total2 = lib().rosaq_plan_schedule(*args, raw, total)
+    assert total2 == total
+    pieces = [dict(zip(PIECE_FIELDS, raw[12 * k:12 * k + 12])) for k in range(total)]
+    return list(begin), pieces
 
 
 class Context:
@@ -215,6 +247,31 @@ class Context:
                "rosaq_linear_multi")
         return outs
 
+    def plan_ctas(self):
+        n = lib().rosaq_plan_ctas(self._h)
+        if n < 0:
+            raise RosaqError(n, "rosaq_plan_ctas")
+        return n
+
+    def plan_create(self, M, ops):
+        """rosaq_plan_create.  ops: list of (x, x_from, handle, y) with x a CUDA fp16 tensor [M][.] or None when
+        x_from >= 0, handle a Rotation or a Weight, y the CUDA fp16 output tensor [M][.]."""
+        arr = (_Op * len(ops))()
+        keep = []
+        for o, (x, x_from, handle, y) in zip(arr, ops):
+            assert y.is_cuda and y.dtype == torch.float16 and y.dim() == 2 and y.stride(1) == 1 and y.shape[0] == M
+            if x is not None:
+                assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1 and x.shape[0] == M
+            o.x, o.ldx = (None if x is None else x.data_ptr()), (0 if x is None else x.stride(0))
+            o.x_from = -1 if x_from is None else int(x_from)
+            o.r = handle._h if isinstance(handle, Rotation) else None
+            o.w = handle._h if isinstance(handle, Weight) else None
+            o.y, o.ldy = y.data_ptr(), y.stride(0)
+            keep += [x, handle, y]
+        h = C.c_void_p()
+        _check(lib().rosaq_plan_create(self._h, int(M), len(ops), arr, C.byref(h)), "rosaq_plan_create")
+        return Plan(self, h, keep)
+
     def linear_static(self, x, weight, rotation=None, out=None, stream=None):
         """rosaq_linear_static: same result as `linear`, but the library allocates nothing (the rotated
         activations live in a fixed 4 MiB array inside the library).  Pass `out`: with out=None this
@@ -264,6 +321,27 @@ class Weight:
             pass
 
 
+class Plan:
+    """rosaq_plan wrapper; keeps the tensors and handles of its operations alive."""
+
+    def __init__(self, ctx, handle, keep):
+        self._ctx, self._h, self._keep = ctx, handle, keep
+
+    def run(self, stream=None):
+        _check(lib().rosaq_plan_run(self._ctx._h, self._h, _stream(stream)), "rosaq_plan_run")
+
+    def free(self):
+        if self._h:
+            lib().rosaq_plan_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
 class Rotation:
     """rosaq_rotation wrapper."""
 
@@ -280,60 +358,3 @@ class Rotation:
             self.free()
         except Exception:
             pass
-
-
-# Module-level spellings with the exact C names.
-def rosaq_create(device=0):
-    return Context(device)
-
-
-def rosaq_destroy(ctx):
-    ctx.close()
-
-
-def rosaq_calib_cov(ctx, X, C_out, n_blocks=1, stream=None):
-    return ctx.calib_cov(X, C_out, n_blocks, stream)
-
-
-def rosaq_quantize(ctx, W, q=None, perm=None, bits=4, group=128, k_salient=128, stream=None):
-    return ctx.quantize(W, q, perm, bits, group, k_salient, stream)
-
-
-def rosaq_weight_export(ctx, weight, stream=None):
-    return weight.export(stream)
-
-
-def rosaq_weight_import(ctx, d_in, d_out, bits, group, k_salient, qw, scales, zeros, salient, stream=None):
-    return ctx.weight_import(d_in, d_out, bits, group, k_salient, qw, scales, zeros, salient, stream)
-
-
-def rosaq_weight_free(weight):
-    weight.free()
-
-
-def rosaq_rotation_create(ctx, q, perm=None, stream=None):
-    return ctx.rotation_create(q, perm, stream)
-
-
-def rosaq_rotation_free(rotation):
-    rotation.free()
-
-
-def rosaq_rotate(ctx, x, rotation, out=None, stream=None):
-    return ctx.rotate(x, rotation, out, stream)
-
-
-def rosaq_linear(ctx, x, weight, rotation=None, out=None, stream=None):
-    return ctx.linear(x, weight, rotation, out, stream)
-
-
-def rosaq_linear_multi(ctx, x, weights, rotation=None, outs=None, stream=None):
-    return ctx.linear_multi(x, weights, rotation, outs, stream)
-
-
-def rosaq_linear_static(ctx, x, weight, rotation=None, out=None, stream=None):
-    return ctx.linear_static(x, weight, rotation, out, stream)
-
-
-def rosaq_last_status(ctx, stream=None):
-    return ctx.last_status(stream)

@@ -68,6 +68,18 @@ int run_gemm(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledO
   return launch_linear_tc(ctx, x, M, ldx, t, col_map, y, ldy, s);
 }
 
+// Up to 64 tokens the default implementation runs everything a call needs -- the rotation and the
+// linears that consume it -- as one persistent launch.
+bool use_plan(const rosaq_ctx *ctx, int M) { return ctx->impl == 0 && M <= 64; }
+
+int run_ops(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, cudaStream_t s) {
+  PlanLaunch l;
+  int st = plan_prepare(ctx, M, n, ops, &l);
+  if (st == ROSAQ_OK) st = plan_launch(ctx, l, s);
+  plan_release(&l);
+  return st;
+}
+
 }  // namespace
 
 extern "C" {
@@ -112,6 +124,11 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->sk_partials = nullptr;
   ctx->sk_arrive = nullptr;
   ctx->sk_ctas = 2 * ctx->sm_count < rosaq::kSkMaxCtas ? 2 * ctx->sm_count : rosaq::kSkMaxCtas;
+  ctx->pl_ctas = 0;
+  ctx->pl_cost[0] = kPlanCostFp16, ctx->pl_cost[1] = kPlanCostQuant, ctx->pl_cost[2] = kPlanCostTile;
+  ctx->pl_partials = nullptr;
+  ctx->pl_partial_bytes = 0;
+  ctx->pl_sync = nullptr;
   st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), sizeof(int)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
   // the stream-K workspace is taken here, once, so that no linear call ever allocates for it
@@ -119,7 +136,17 @@ int rosaq_create(rosaq_ctx **out, int device) {
     st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->sk_partials), (size_t)ctx->sk_ctas * 2 * rosaq::kSkPartialBytes));
   if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->sk_arrive), rosaq::kSkCounterInts * sizeof(int)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->pl_sync), rosaq::kPlSyncWords * sizeof(unsigned)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->pl_sync, 0, rosaq::kPlSyncWords * sizeof(unsigned)));
+  // the partial tiles of a launch whose CTAs all share tiles at both ends of two phases (grown if a plan needs more)
+  if (st == ROSAQ_OK) {
+    const size_t bytes = (size_t)4 * ctx->sk_ctas * rosaq::kSkPartialBytes;
+    st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->pl_partials), bytes));
+    if (st == ROSAQ_OK) ctx->pl_partial_bytes = bytes;
+  }
   if (st != ROSAQ_OK) {
+    if (ctx->pl_sync) (void)cudaFree(ctx->pl_sync);
+    if (ctx->pl_partials) (void)cudaFree(ctx->pl_partials);
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
     if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
     if (ctx->sk_arrive) (void)cudaFree(ctx->sk_arrive);
@@ -139,6 +166,9 @@ int rosaq_destroy(rosaq_ctx *ctx) {
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
     if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
     if (ctx->sk_arrive) (void)cudaFree(ctx->sk_arrive);
+    if (ctx->pl_sync) (void)cudaFree(ctx->pl_sync);
+    if (ctx->pl_partials) (void)cudaFree(ctx->pl_partials);
+    plan_free_schedules(ctx);
     (void)cudaGetLastError();
   }
   delete ctx;
@@ -160,6 +190,8 @@ int rosaq_last_status(rosaq_ctx *ctx, void *stream) {
     if (st != ROSAQ_OK) return st;
     // a launch that gave up may have left arrival counters of the stream-K exchange behind
     st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
+    if (st != ROSAQ_OK) return st;
+    st = cuda_status(cudaMemset(ctx->pl_sync, 0, rosaq::kPlSyncWords * sizeof(unsigned)));
     if (st != ROSAQ_OK) return st;
   }
   return host;
@@ -363,6 +395,10 @@ int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
   if (st != ROSAQ_OK) return st;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return ROSAQ_ERR_CUDA;
+  if (use_plan(ctx, M)) {
+    const PlanOp op{static_cast<const __half *>(x), ldx, -1, &r->t, r->col_map, static_cast<__half *>(x_rot), ldxr};
+    return run_ops(ctx, M, 1, &op, static_cast<cudaStream_t>(stream));
+  }
   return run_gemm(ctx, static_cast<const __half *>(x), M, ldx, r->t, r->col_map, static_cast<__half *>(x_rot), ldxr,
                   static_cast<cudaStream_t>(stream));
 }
@@ -382,6 +418,16 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
   if (r) {
     st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
     if (st != ROSAQ_OK) return st;
+  }
+  if (use_plan(ctx, M)) {
+    // one launch: x . R into the workspace (phase 1), the GEMM stage on it (phase 2)
+    PlanOp ops[2];
+    int n = 0;
+    if (r) ops[n++] = PlanOp{xin, ldx, -1, &r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d};
+    ops[n] = PlanOp{xin, ldx, r ? 0 : -1, &w->t, nullptr, static_cast<__half *>(y), ldy};
+    return run_ops(ctx, M, n + 1, ops, s);
+  }
+  if (r) {
     st = run_gemm(ctx, xin, M, ldx, r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d, s);
     if (st != ROSAQ_OK) return st;
     xin = static_cast<const __half *>(ctx->ws);
@@ -412,6 +458,15 @@ int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const 
   if (r) {
     st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
     if (st != ROSAQ_OK) return st;
+  }
+  if (use_plan(ctx, M)) {
+    PlanOp ops[5];
+    int k = 0;
+    if (r) ops[k++] = PlanOp{xin, ldx, -1, &r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d};
+    for (int i = 0; i < n; ++i) ops[k++] = PlanOp{xin, ldx, r ? 0 : -1, &w[i]->t, nullptr, static_cast<__half *>(y[i]), ldy[i]};
+    return run_ops(ctx, M, k, ops, s);
+  }
+  if (r) {
     st = run_gemm(ctx, xin, M, ldx, r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d, s);
     if (st != ROSAQ_OK) return st;
     xin = static_cast<const __half *>(ctx->ws);
@@ -427,6 +482,94 @@ int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const 
   long long ldys[4];
   for (int i = 0; i < n; ++i) ts[i] = &w[i]->t, ys[i] = static_cast<__half *>(y[i]), ldys[i] = ldy[i];
   return launch_linear_tc_multi(ctx, xin, M, ld, n, ts, nullptr, ys, ldys, s);
+}
+
+int rosaq_plan_create(rosaq_ctx *ctx, int M, int n_ops, const rosaq_op *ops, rosaq_plan **out) {
+  if (!out) return ROSAQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !ops || n_ops < 1 || M < 1) return ROSAQ_ERR_INVALID_ARG;
+  if (n_ops > kPlanMaxOps || M > 64) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  rosaq_plan *pl = new (std::nothrow) rosaq_plan();
+  if (!pl) return ROSAQ_ERR_ALLOC;
+  pl->M = M;
+  pl->device = ctx->device;
+  int st = ROSAQ_OK;
+  for (int i = 0; i < n_ops && st == ROSAQ_OK; ++i) {
+    const rosaq_op &o = ops[i];
+    if ((o.r != nullptr) == (o.w != nullptr) || o.x_from >= i) {
+      st = ROSAQ_ERR_INVALID_ARG;
+      break;
+    }
+    const TiledOperand &t = o.r ? o.r->t : o.w->t;
+    const void *x = o.x_from >= 0 ? ops[o.x_from].y : o.x;
+    const int64_t ldx = o.x_from >= 0 ? ops[o.x_from].ldy : o.ldx;
+    if (o.x_from >= 0) {
+      const rosaq_op &src = ops[o.x_from];
+      const int src_d_out = src.r ? src.r->t.d_out : src.w->t.d_out;
+      if (src_d_out != t.d_in) st = ROSAQ_ERR_INVALID_ARG;
+    }
+    if (st == ROSAQ_OK) st = check_act(x, M, ldx, t.d_in);
+    if (st == ROSAQ_OK) st = check_act(o.y, M, o.ldy, t.d_out);
+    if (st == ROSAQ_OK && (o.r ? o.r->device : o.w->device) != ctx->device) st = ROSAQ_ERR_INVALID_ARG;
+    if (st == ROSAQ_OK)
+      pl->ops.push_back(PlanOp{static_cast<const __half *>(x), ldx, o.x_from >= 0 ? o.x_from : -1, &t,
+                               o.r ? o.r->col_map : nullptr, static_cast<__half *>(o.y), o.ldy});
+  }
+  if (st == ROSAQ_OK) {
+    DeviceGuard guard(ctx->device);
+    st = guard.ok ? plan_prepare(ctx, M, n_ops, pl->ops.data(), &pl->launch) : ROSAQ_ERR_CUDA;
+  }
+  if (st != ROSAQ_OK) {
+    delete pl;
+    return st;
+  }
+  *out = pl;
+  return ROSAQ_OK;
+}
+
+int rosaq_plan_run(rosaq_ctx *ctx, const rosaq_plan *plan, void *stream) {
+  if (!ctx || !plan || plan->device != ctx->device) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  return plan_launch(ctx, plan->launch, static_cast<cudaStream_t>(stream));
+}
+
+int rosaq_plan_free(rosaq_plan *plan) {
+  if (!plan) return ROSAQ_ERR_INVALID_ARG;
+  plan_release(&plan->launch);
+  delete plan;
+  return ROSAQ_OK;
+}
+
+int rosaq_plan_ctas(rosaq_ctx *ctx) {
+  if (!ctx) return ROSAQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return ROSAQ_ERR_CUDA;
+  const int p = plan_ctas(ctx);
+  return p > 0 ? p : ROSAQ_ERR_CUDA;
+}
+
+int rosaq_plan_schedule(int n_ops, const int32_t *n_tiles, const int32_t *groups, const int32_t *g_fp16, const int32_t *x_from,
+                        const int32_t *copies, int n_ctas, int32_t *piece_begin, int32_t *pieces, int max_pieces) {
+  if (n_ops < 1 || n_ops > kPlanMaxOps || !n_tiles || !groups || !g_fp16 || !x_from || n_ctas < 1 || !piece_begin ||
+      (!pieces && max_pieces > 0) || max_pieces < 0)
+    return ROSAQ_ERR_INVALID_ARG;
+  std::vector<PlanGeom> geom(n_ops);
+  for (int i = 0; i < n_ops; ++i) geom[i] = PlanGeom{n_tiles[i], groups[i], g_fp16[i], x_from[i] < 0 ? -1 : x_from[i], copies ? copies[i] : 1,
+                       copies && copies[i] > 1 ? kPlanCostScatterTile : 0};
+  const int cost[3] = {kPlanCostFp16, kPlanCostQuant, kPlanCostTile};
+  PlanSchedule s;
+  const int st = plan_build_schedule(geom, n_ctas, cost, &s);
+  if (st != ROSAQ_OK) return st;
+  for (int c = 0; c <= n_ctas; ++c) piece_begin[c] = s.seg_begin[c];
+  const int total = (int)s.segs.size();
+  for (int k = 0; k < total && k < max_pieces; ++k) {
+    const PlanSeg &g = s.segs[k];
+    int32_t *o = pieces + (size_t)k * 12;
+    o[0] = g.prob, o[1] = g.tile, o[2] = g.g_begin, o[3] = g.g_end, o[4] = g.n_contrib, o[5] = g.contrib_idx;
+    o[6] = g.slot0, o[7] = g.counter, o[8] = g.closer_idx, o[9] = g.n_closers, o[10] = g.tok_begin, o[11] = g.tok_end;
+  }
+  return total;
 }
 
 }  // extern "C"

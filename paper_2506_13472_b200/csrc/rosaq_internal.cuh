@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "rosaq.h"
 
 namespace rosaq {
@@ -167,6 +169,64 @@ namespace rosaq {
 constexpr int kSkMaxCtas = 320;                     // stream-K grid limit (two CTAs per SM)
 constexpr int kSkCounterInts = 1024;                // arrival counters (one per column tile of a launch)
 constexpr size_t kSkPartialBytes = 128 * 64 * sizeof(float);   // one partial tile: 128 columns x 64 tokens
+
+// ---- the persistent multi-problem launch (linear_plan.cu) --------------------------------
+constexpr int kPlanMaxOps = 12;                     // problems in one launch
+constexpr int kPlanMaxCtas = 512;
+constexpr int kPlMaxCounters = 4096;                // column tiles shared between CTAs in one launch
+constexpr int kPlSyncFinished = 0, kPlSyncDone = 4, kPlSyncArrive = 16;   // word offsets in the sync buffer
+constexpr int kPlSyncWords = kPlSyncArrive + kPlMaxCounters;
+// Relative cost of the work items when a phase is cut into equal shares: an fp16 group is bound by its
+// 32 KB of HBM traffic (about 1400 cycles of an SM's share of the bandwidth), a quantized one by its eight
+// MMAs (about 420 cycles), and every tile a CTA starts costs a little for switching accumulators.
+constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 3, kPlanCostTile = 1, kPlanCostScatterTile = 48;
+
+// One piece of work of a CTA: groups [g_begin, g_end) of column tile `tile` of problem `prob`.
+struct PlanSeg {
+  int prob, tile, g_begin, g_end;
+  int n_contrib;        // CTAs that hold groups of this tile (1: the tile is this CTA's alone)
+  int contrib_idx;      // this CTA's position among them, ascending K
+  int slot0;            // partial-tile slot of holder 0; holder i uses slot0 + i
+  int counter;          // the tile's arrival counter
+  int closer_idx;       // >= 0: this CTA adds the partial tiles for token rows closer_idx, + n_closers, ...
+  int n_closers;
+  int tok_begin, tok_end;   // token rows of y this piece writes when it finishes the tile (a whole tile: all)
+};
+static_assert(sizeof(PlanSeg) == 48, "three 16-byte loads per piece");
+
+struct PlanGeom {
+  int n_tiles, groups, g_fp16;
+  int dep;              // index of the problem whose output this one reads, or -1
+  int rep;              // >= 1: every tile is computed `rep` times, each copy writing 1/rep of the token rows
+  int tile_cost;        // cost of starting a tile (copy) of this problem; 0: the default
+};
+
+struct PlanSchedule {
+  std::vector<PlanGeom> geom;
+  int cost[3];
+  int n_ctas = 0, n_counters = 0, n_slots = 0;
+  std::vector<PlanSeg> segs;          // per CTA, in processing order
+  std::vector<int> seg_begin;         // [n_ctas + 1]
+  std::vector<unsigned> done_target;  // per problem: finishing events that complete it
+  PlanSeg *d_segs = nullptr;
+  int *d_seg_begin = nullptr;
+};
+
+struct PlanOp {
+  const __half *x;      // input activations (ignored when dep >= 0)
+  long long ldx;
+  int dep;              // >= 0: the input is the output of that earlier op
+  const TiledOperand *t;
+  const int32_t *col_map;
+  __half *y;
+  long long ldy;
+};
+
+struct PlanLaunch {
+  void *params = nullptr;   // kernel parameters (tensor maps, problem table), owned
+  int n_ctas = 0, bits = 4;
+  size_t partial_bytes = 0;
+};
 }  // namespace rosaq
 
 struct rosaq_ctx {
@@ -180,11 +240,24 @@ struct rosaq_ctx {
   float *sk_partials;  // stream-K: fp32 partial tiles, [sk_ctas][2][64 tokens][128 columns]
   int *sk_arrive;      // stream-K: per-tile arrival counters, zero between launches
   int sk_ctas;         // CTAs the partial-tile workspace was sized for
+  // persistent multi-problem launch
+  int pl_ctas;                                   // CTAs of its grid (0 until first asked for)
+  int pl_cost[3];                                // cost of an fp16 group, a quantized group, a tile's epilogue
+  float *pl_partials;                            // partial tiles exchanged between CTAs; grown on demand
+  size_t pl_partial_bytes;
+  unsigned *pl_sync;                             // counters, zero between launches
+  std::vector<rosaq::PlanSchedule *> pl_schedules;   // one per geometry seen, owned
 };
 
 struct rosaq_weight {
   rosaq::TiledOperand t;
   int group, k_salient, device;
+};
+
+struct rosaq_plan {
+  std::vector<rosaq::PlanOp> ops;
+  int M, device;
+  rosaq::PlanLaunch launch;
 };
 
 struct rosaq_rotation {
@@ -232,5 +305,12 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
 int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, int n,
                            const TiledOperand *const *ts, const int32_t *col_map, __half *const *ys,
                            const long long *ldys, cudaStream_t s);
+
+int plan_build_schedule(const std::vector<PlanGeom> &ops, int n_ctas, const int *cost, PlanSchedule *out);
+int plan_ctas(rosaq_ctx *ctx);
+int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *out);
+int plan_launch(rosaq_ctx *ctx, const PlanLaunch &l, cudaStream_t s);
+void plan_release(PlanLaunch *l);
+void plan_free_schedules(rosaq_ctx *ctx);
 
 }  // namespace rosaq
