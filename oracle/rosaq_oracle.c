@@ -18,10 +18,12 @@
  *
  * Parity status.  Pinned by identities / library routines / brute force in the
  * CPU tests: cov (Eq. 4), eigh_jacobi (Eq. 4), rotate_weights_f64 (Eq. 1),
- * forward (Eq. 1, Eq. 3, Eq. 6 vs Eq. 7), f16 conversions, pack/unpack.
+ * scale_rows (scaling invariance), forward (Eq. 1, Eq. 3, Eq. 6 vs Eq. 7),
+ * f16 conversions, pack/unpack.
  * The quantizer's free constants (range floor 1e-5, zero-point clamp, tie rule,
  * scale rounded to fp16 before the codes are taken), the bit layout of the packed
- * words and the fp32 summation order of rotate_weights_f32 are NOT fixed by the
+ * words, the fp32 summation order of rotate_weights_f32 and the choice of the
+ * diagonal D of the scaled (AWQ-style) variant are NOT fixed by the
  * paper: for those this file is the definition ("parity unpinned" by the paper);
  * the tests pin their internal consistency (grid round trip, error bound,
  * bijection) only.
@@ -240,18 +242,13 @@ void oracle_rotate_weights_f64(const double *Rb, int d_in, int n_blocks, const i
   }
 }
 
-/* The canonical fp32 version whose result defines the integer codes: one fused
+/* The canonical fp32 chain whose result defines the integer codes: one fused
  * multiply-add per term, k ascending, a single accumulator started at +0, no
- * blocking and no reassociation.  R is fp32, W is binary16 (widened exactly). */
-void oracle_rotate_weights_f32(const float *Rb, int d_in, int n_blocks, const int32_t *perm,
-                               const uint16_t *W16, int d_out, const int32_t *cols, int n_cols,
-                               float *out) {
+ * blocking and no reassociation.  Wc holds the needed columns of W in fp32:
+ * Wc[k][ci]. */
+static void rotate_chain_f32(const float *Rb, int d_in, int n_blocks, const int32_t *perm,
+                             const float *Wc, int n_cols, float *out) {
   int dh = d_in / n_blocks;
-  /* widen the needed columns of W once: Wc[k][ci] */
-  float *Wc = (float *)malloc(sizeof(float) * (size_t)d_in * n_cols);
-  for (int k = 0; k < d_in; ++k)
-    for (int ci = 0; ci < n_cols; ++ci)
-      Wc[(int64_t)k * n_cols + ci] = (float)f16_bits_to_double(W16[(int64_t)k * d_out + cols[ci]]);
 #pragma omp parallel for schedule(static)
   for (int j = 0; j < d_in; ++j) {
     int p = perm ? perm[j] : j;
@@ -264,7 +261,50 @@ void oracle_rotate_weights_f32(const float *Rb, int d_in, int n_blocks, const in
       out[(int64_t)j * n_cols + ci] = acc;
     }
   }
+}
+
+/* R is fp32, W is binary16 (widened exactly). */
+void oracle_rotate_weights_f32(const float *Rb, int d_in, int n_blocks, const int32_t *perm,
+                               const uint16_t *W16, int d_out, const int32_t *cols, int n_cols,
+                               float *out) {
+  float *Wc = (float *)malloc(sizeof(float) * (size_t)d_in * n_cols);
+  for (int k = 0; k < d_in; ++k)
+    for (int ci = 0; ci < n_cols; ++ci)
+      Wc[(int64_t)k * n_cols + ci] = (float)f16_bits_to_double(W16[(int64_t)k * d_out + cols[ci]]);
+  rotate_chain_f32(Rb, d_in, n_blocks, perm, Wc, n_cols, out);
   free(Wc);
+}
+
+/* The same chain on a weight that is already fp32 (the scaled weight D W below). */
+void oracle_rotate_weights_f32_w32(const float *Rb, int d_in, int n_blocks, const int32_t *perm,
+                                   const float *W32, int d_out, const int32_t *cols, int n_cols,
+                                   float *out) {
+  float *Wc = (float *)malloc(sizeof(float) * (size_t)d_in * n_cols);
+  for (int k = 0; k < d_in; ++k)
+    for (int ci = 0; ci < n_cols; ++ci) Wc[(int64_t)k * n_cols + ci] = W32[(int64_t)k * d_out + cols[ci]];
+  rotate_chain_f32(Rb, d_in, n_blocks, perm, Wc, n_cols, out);
+  free(Wc);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Scaling invariance (appendix on rotational and scaling invariance):          */
+/*   X W = (X D^-1)(D W)  for an invertible diagonal D, so a linear layer may    */
+/* quantize D W and be fed X D^-1.  The weight-splitting appendix uses this      */
+/* (AWQ-style per-input-channel scaling) for the down projection W_D, which it   */
+/* does not rotate.  The paper prints no rule for D: D is an input here.         */
+/*   out[i][n] = d[i] * W[i][n]                                                  */
+/* fp64 for the identity checks; fp32 (binary16 weight widened exactly, one      */
+/* rounding per product) for the version the integer codes are taken from.       */
+/* ------------------------------------------------------------------------- */
+void oracle_scale_rows_f64(const double *W, int d_in, int d_out, const double *d, double *out) {
+  for (int i = 0; i < d_in; ++i)
+    for (int n = 0; n < d_out; ++n) out[(int64_t)i * d_out + n] = d[i] * W[(int64_t)i * d_out + n];
+}
+
+void oracle_scale_rows_f32(const uint16_t *W16, int d_in, int d_out, const float *d, float *out) {
+  for (int i = 0; i < d_in; ++i)
+    for (int n = 0; n < d_out; ++n)
+      out[(int64_t)i * d_out + n] = d[i] * (float)f16_bits_to_double(W16[(int64_t)i * d_out + n]);
 }
 
 /* ------------------------------------------------------------------------- */

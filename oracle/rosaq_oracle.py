@@ -141,17 +141,37 @@ def rotate_weights_f64(Rb, W, perm=None, cols=None):
     return out
 
 
-def rotate_weights_f32(Rb32, W16, perm=None, cols=None):
-    """The canonical fp32 fused-multiply-add chain (k ascending) that defines the codes."""
+def rotate_weights_f32(Rb32, W, perm=None, cols=None):
+    """The canonical fp32 fused-multiply-add chain (k ascending) that defines the codes.
+    W is the binary16 weight, or an fp32 array (the scaled weight D W of scale_rows_f32)."""
     Rb = _blocks(Rb32, np.float32)
-    W16 = _c(W16, np.float16)
-    d_in, d_out = W16.shape
+    w32 = np.asarray(W).dtype == np.float32
+    W = _c(W, np.float32 if w32 else np.float16)
+    d_in, d_out = W.shape
     cols = np.arange(d_out, dtype=np.int32) if cols is None else _c(cols, np.int32)
     perm = None if perm is None else _c(perm, np.int32)
     out = np.empty((d_in, cols.size), np.float32)
-    _L().oracle_rotate_weights_f32(_p(Rb), C.c_int(d_in), C.c_int(Rb.shape[0]), _p(perm),
-                                   _p(W16.view(np.uint16)), C.c_int(d_out), _p(cols),
-                                   C.c_int(cols.size), _p(out))
+    fn = _L().oracle_rotate_weights_f32_w32 if w32 else _L().oracle_rotate_weights_f32
+    fn(_p(Rb), C.c_int(d_in), C.c_int(Rb.shape[0]), _p(perm), _p(W if w32 else W.view(np.uint16)), C.c_int(d_out),
+       _p(cols), C.c_int(cols.size), _p(out))
+    return out
+
+
+def scale_rows_f64(W, d):
+    """D W in fp64 (scaling invariance: X W = (X D^-1)(D W))."""
+    W64 = f16_to_f64(W) if np.asarray(W).dtype == np.float16 else _c(W, np.float64)
+    d = _c(d, np.float64)
+    out = np.empty(W64.shape, np.float64)
+    _L().oracle_scale_rows_f64(_p(W64), C.c_int(W64.shape[0]), C.c_int(W64.shape[1]), _p(d), _p(out))
+    return out
+
+
+def scale_rows_f32(W16, d32):
+    """D W in fp32, one rounding per product: the weight the scaled variant quantizes."""
+    W16 = _c(W16, np.float16)
+    d = _c(d32, np.float32)
+    out = np.empty(W16.shape, np.float32)
+    _L().oracle_scale_rows_f32(_p(W16.view(np.uint16)), C.c_int(W16.shape[0]), C.c_int(W16.shape[1]), _p(d), _p(out))
     return out
 
 

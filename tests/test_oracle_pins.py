@@ -407,3 +407,79 @@ def test_frozen_quantizer_output_has_not_drifted():
         assert list(qd["salient"].view(np.uint16)[0]) == want[b]["salient_row0"]
         for r in range(qw.shape[0]):
             assert list(qw[r]) == want[b][f"qw{r}"]
+
+
+# --------------------------------------------------------------------------- scaling invariance (W_D variant)
+def test_scaling_invariance_fp64_with_and_without_rotation():
+    """X W = (X D^-1)(D W) for any invertible diagonal D (appendix on rotational and scaling invariance),
+    alone and combined with an orthogonal R: (X D^-1 R)(R^T D W) = X W, <= 1e-10 in fp64."""
+    rng = np.random.default_rng(31)
+    d_in, d_out, M = 256, 24, 5
+    W = rng.standard_normal((d_in, d_out))
+    x = rng.standard_normal((M, d_in))
+    d = rng.uniform(0.25, 4.0, d_in)
+    ref = x @ W
+    DW = orc.scale_rows_f64(W, d)
+    assert np.array_equal(DW[7], d[7] * W[7])                              # row i scaled by d[i], nothing else
+    assert np.linalg.norm((x / d) @ DW - ref) / np.linalg.norm(ref) <= 1e-10
+    R = synth.orthogonal_qr(d_in, rng)
+    Wp = orc.rotate_weights_f64(R, DW)
+    assert np.linalg.norm(((x / d) @ R) @ Wp - ref) / np.linalg.norm(ref) <= 1e-10
+    # a wrong side (D applied to the columns, or D^-1 forgotten) must not pass
+    assert np.linalg.norm(x @ DW - ref) / np.linalg.norm(ref) > 1e-2
+
+
+def test_scale_rows_f32_is_one_rounded_product_and_identity_for_ones():
+    rng = np.random.default_rng(32)
+    W = (rng.standard_normal((8, 6)) * 0.02).astype(np.float16)
+    ones = np.ones(8, np.float32)
+    assert np.array_equal(orc.scale_rows_f32(W, ones).view(np.uint32), W.astype(np.float32).view(np.uint32))
+    d = np.array([0.5, 2.0, 3.0, 1.0 / 3.0, 0.1, 7.0, 1e-3, 1.5], np.float32)
+    got = orc.scale_rows_f32(W, d)
+    for i in range(8):
+        for n in range(6):
+            want = _round_f32(Fraction(float(d[i])) * Fraction(float(W[i, n])))
+            assert got[i, n].view(np.uint32) == want.view(np.uint32)
+    # exactly representable products: 0.75 * 3 = 2.25, 0.375 * 0.5 = 0.1875
+    Wk = np.array([[0.75], [0.375]], np.float16)
+    assert orc.scale_rows_f32(Wk, np.array([3.0, 0.5], np.float32)).tolist() == [[2.25], [0.1875]]
+
+
+def test_scaled_quantization_hand_computed_group_and_unit_scale_is_todays_path():
+    """A group whose rows are 0, 1, ..., 127 times 2^-10 scaled by D = 2 quantizes like the group 0 .. 127 times
+    2^-9 (INT4: range 127 * 2^-9, fifteen steps); with D = 1 every output bit equals the unscaled path."""
+    rows = (np.arange(128, dtype=np.float64) * 2.0 ** -10)
+    W = np.concatenate([np.zeros((128, 1)), rows[:, None]], axis=0).astype(np.float16)      # salient group + one group
+    two = np.full(256, 2.0, np.float32)
+    a = orc.quantize(orc.scale_rows_f32(W, two), 4, 128, 128)
+    b = orc.quantize((W.astype(np.float32) * np.float32(2.0)), 4, 128, 128)
+    for k in ("salient", "scales", "zeros", "codes"):
+        assert np.array_equal(a[k], b[k])
+    s = np.float16(np.float32(127 * 2.0 ** -9) / np.float32(15))
+    assert a["scales"][0, 0] == s and a["zeros"][0, 0] == 0
+    assert a["codes"][0, 0] == 0 and a["codes"][127, 0] == 15
+    assert a["codes"][64, 0] == int(np.rint(np.float32(64 * 2.0 ** -9) / np.float32(s)))
+    one = np.ones(256, np.float32)
+    c = orc.quantize(orc.scale_rows_f32(W, one), 4, 128, 128)
+    e = orc.quantize(W.astype(np.float32), 4, 128, 128)
+    for k in ("salient", "scales", "zeros", "codes"):
+        assert np.array_equal(c[k], e[k])
+
+
+def test_scaled_then_rotated_chain_takes_the_fp32_scaled_weight():
+    rng = np.random.default_rng(33)
+    d_in, d_out = 64, 5
+    W = (rng.standard_normal((d_in, d_out)) * 0.02).astype(np.float16)
+    R = synth.orthogonal_qr(d_in, rng).astype(np.float32)
+    d = rng.uniform(0.5, 2.0, d_in).astype(np.float32)
+    DW = orc.scale_rows_f32(W, d)
+    got = orc.rotate_weights_f32(R, DW)
+    for i in (0, 17, 63):
+        for n in range(d_out):
+            acc = np.float32(0.0)
+            for k in range(d_in):
+                acc = _round_f32(Fraction(float(R[k, i])) * Fraction(float(DW[k, n])) + Fraction(float(acc)))
+            assert got[i, n].view(np.uint32) == acc.view(np.uint32)
+    # and it is the same chain as the binary16 entry when the scaled weight happens to be the widened one
+    assert np.array_equal(orc.rotate_weights_f32(R, W.astype(np.float32)).view(np.uint32),
+                          orc.rotate_weights_f32(R, W).view(np.uint32))
