@@ -140,7 +140,9 @@ int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens
  * ascending, so that its bits (and therefore every code) are reproducible.
  * Rows [0, k_salient) of W' are rounded to fp16 and kept; every further group of
  * 128 rows is quantized per output column with asymmetric min/max round-to-nearest:
- *   s = fp16(max(hi-lo, 1e-5) / (2^bits-1)), z = clamp(-rint(lo/s), 0, 2^bits-1),
+ *   s = fp16(max(hi-lo, 1e-5) / (2^bits-1)), with an fp16 result of zero replaced by the smallest
+ *       subnormal (bits 0x0001) and an infinite one by the largest finite value (0x7bff),
+ *   z = clamp(-rint(lo/s), 0, 2^bits-1), stored as +0 when lo >= 0,
  *   code = clamp(rint(w/s) + z, 0, 2^bits-1), all IEEE fp32, ties to even.
  * Allocates the result (*out, release with rosaq_weight_free) and a temporary fp32
  * W' of d_in*d_out floats that is freed before returning.  Synchronizes `stream`.
@@ -148,6 +150,19 @@ int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens
  */
 int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot,
                    int bits, int group, int k_salient, rosaq_weight **out, void *stream);
+
+/*
+ * The same for the scaled weight D W (scaling invariance, X W = (X D^-1)(D W); the weight-splitting appendix
+ * quantizes the down projection W_D this way, AWQ-style, without rotating it):
+ *   in_scale  DEVICE fp32 [d_in], the diagonal of D; NULL = rosaq_quantize.  The paper gives no rule for D:
+ *             it is an input, like R; the caller feeds rosaq_linear the activations x D^-1 (R).
+ * W'' = R^T (D W): each product d[i] * W[i][n] is rounded once to fp32, then the chain of rosaq_quantize runs
+ * on those values (rot == NULL: W'' = D W).  With rot and in_scale both given a second temporary of
+ * d_in*d_out floats is allocated and freed.  Everything else as rosaq_quantize.
+ */
+int rosaq_quantize_scaled(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot,
+                          const float *in_scale, int bits, int group, int k_salient, rosaq_weight **out,
+                          void *stream);
 
 /*
  * Interchange layout of a quantized weight (r = row index inside the non-salient part):
@@ -247,7 +262,13 @@ int rosaq_plan_create(rosaq_ctx *ctx, int M, int n_ops, const rosaq_op *ops, ros
 int rosaq_plan_run(rosaq_ctx *ctx, const rosaq_plan *plan, void *stream);
 int rosaq_plan_free(rosaq_plan *plan);
 
-/* Number of CTAs of the persistent launch on the context's device (two per SM), or a negative status. */
+/* Test and tuning hook: the relative cost of an fp16 group, a quantized group and a started tile that
+ * rosaq_plan_create (and the single calls, which plan internally) use from now on to cut a phase into
+ * equal shares (defaults 10, 7, 1; 1 <= cost <= 1000, tile >= 0).  Changes how K is divided among the CTAs,
+ * hence the fp32 summation order of later plans; plans already created keep theirs. */
+int rosaq_set_plan_costs(rosaq_ctx *ctx, int fp16_group, int quant_group, int tile);
+
+/* Number of CTAs of the persistent launch on the context's device (one per SM), or a negative status. */
 int rosaq_plan_ctas(rosaq_ctx *ctx);
 
 /*

@@ -19,11 +19,11 @@ ROSAQ_ERR_ALLOC, ROSAQ_ERR_CUDA, ROSAQ_ERR_TIMEOUT, ROSAQ_ERR_UNSUPPORTED_ARCH =
 
 EXPORTS = [
     "rosaq_create", "rosaq_destroy", "rosaq_strerror", "rosaq_last_status", "rosaq_set_wait_limit",
-    "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_weight_export",
+    "rosaq_set_linear_impl", "rosaq_calib_cov", "rosaq_quantize", "rosaq_quantize_scaled", "rosaq_weight_export",
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
     "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_multi", "rosaq_linear_static",
     "rosaq_plan_equal_shares", "rosaq_plan_create", "rosaq_plan_run", "rosaq_plan_free", "rosaq_plan_ctas",
-    "rosaq_plan_schedule",
+    "rosaq_plan_schedule", "rosaq_set_plan_costs",
 ]
 
 
@@ -65,6 +65,8 @@ def lib():
                                       C.c_void_p, C.c_void_p]
         L.rosaq_quantize.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.POINTER(_Rot), C.c_int, C.c_int,
                                      C.c_int, C.POINTER(C.c_void_p), C.c_void_p]
+        L.rosaq_quantize_scaled.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.POINTER(_Rot), C.c_void_p, C.c_int,
+                                            C.c_int, C.c_int, C.POINTER(C.c_void_p), C.c_void_p]
         L.rosaq_weight_export.argtypes = [C.c_void_p] * 7
         L.rosaq_weight_import.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]
@@ -84,6 +86,7 @@ def lib():
         L.rosaq_plan_run.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.rosaq_plan_free.argtypes = [C.c_void_p]
         L.rosaq_plan_ctas.argtypes = [C.c_void_p]
+        L.rosaq_set_plan_costs.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
         L.rosaq_plan_schedule.argtypes = [C.c_int] + [C.POINTER(C.c_int32)] * 5 + [C.c_int, C.POINTER(C.c_int32),
                                                                                   C.POINTER(C.c_int32), C.c_int]
         _lib = L
@@ -193,13 +196,20 @@ class Context:
         return C_out
 
     # -- Eq. 3
-    def quantize(self, W, q=None, perm=None, bits=4, group=128, k_salient=128, stream=None):
+    def quantize(self, W, q=None, perm=None, bits=4, group=128, k_salient=128, stream=None, in_scale=None):
+        """rosaq_quantize, or rosaq_quantize_scaled when in_scale (fp32 CUDA tensor [d_in]) is given."""
         assert W.is_cuda and W.dtype == torch.float16 and W.is_contiguous() and W.dim() == 2
         rot = None if q is None else _rot_struct(q, perm)
         h = C.c_void_p()
-        _check(lib().rosaq_quantize(self._h, _ptr(W), W.shape[0], W.shape[1],
-                                    None if rot is None else C.byref(rot), bits, group, k_salient, C.byref(h),
-                                    _stream(stream)), "rosaq_quantize")
+        if in_scale is None:
+            _check(lib().rosaq_quantize(self._h, _ptr(W), W.shape[0], W.shape[1],
+                                        None if rot is None else C.byref(rot), bits, group, k_salient, C.byref(h),
+                                        _stream(stream)), "rosaq_quantize")
+        else:
+            assert in_scale.is_cuda and in_scale.dtype == torch.float32 and in_scale.numel() == W.shape[0]
+            _check(lib().rosaq_quantize_scaled(self._h, _ptr(W), W.shape[0], W.shape[1],
+                                               None if rot is None else C.byref(rot), _ptr(in_scale.contiguous()), bits, group,
+                                               k_salient, C.byref(h), _stream(stream)), "rosaq_quantize_scaled")
         return Weight(self, h)
 
     def weight_import(self, d_in, d_out, bits, group, k_salient, qw, scales, zeros, salient, stream=None):
@@ -246,6 +256,9 @@ class Context:
                                         None if rotation is None else rotation._h, n, wa, ya, la, _stream(stream)),
                "rosaq_linear_multi")
         return outs
+
+    def set_plan_costs(self, fp16_group, quant_group, tile):
+        _check(lib().rosaq_set_plan_costs(self._h, fp16_group, quant_group, tile), "rosaq_set_plan_costs")
 
     def plan_ctas(self):
         n = lib().rosaq_plan_ctas(self._h)

@@ -482,37 +482,30 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       epi_bar();
       if (ab.set()) break;
       {
-        // (the two warps of a quadrant take alternate batches of four rows)
+        // (the two warps of a quadrant take alternate batches of eight rows; 32 loads are in flight per
+        // thread and round; a holder index past S adds +0, which changes nothing)
         const int nc = s.n_closers;
         const int t0 = s.tok_begin, t1 = s.tok_end < p.M ? s.tok_end : p.M;
-        for (int r0 = s.closer_idx + ((warp - kPlFirstEpiWarp) >> 2) * 4 * nc; r0 < t1; r0 += 8 * nc) {
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          int i = 0;
-          for (; i + 4 <= S; i += 4) {
-            float w[4][4];
+        for (int r0 = s.closer_idx + ((warp - kPlFirstEpiWarp) >> 2) * 8 * nc; r0 < t1; r0 += 16 * nc) {
+          float acc[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < 8; ++u) acc[u] = 0.f;
+          for (int i = 0; i < S; i += 4) {
+            float w[8][4];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
               const int r = r0 + u * nc;
 #pragma unroll
-              for (int k = 0; k < 4; ++k) w[u][k] = r < t1 ? __ldcg(src0 + (long long)(i + k) * p.slot_floats + r * kTileN) : 0.f;
+              for (int k = 0; k < 4; ++k)
+                w[u][k] = (r < t1 && i + k < S) ? __ldcg(src0 + (long long)(i + k) * p.slot_floats + r * kTileN) : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < 8; ++u)
 #pragma unroll
               for (int k = 0; k < 4; ++k) acc[u] = __fadd_rn(acc[u], w[u][k]);
           }
-          for (; i < S; ++i) {
-            float w[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int r = r0 + u * nc;
-              w[u] = r < t1 ? __ldcg(src0 + (long long)i * p.slot_floats + r * kTileN) : 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) acc[u] = __fadd_rn(acc[u], w[u]);
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < 8; ++u) {
             const int r = r0 + u * nc;
             if (n_ok && r >= t0 && r < t1) y_out[(long long)r * ldy + out_col] = __float2half_rn(acc[u]);
           }

@@ -100,10 +100,10 @@ gemm_tn_fma_kernel(const TA *__restrict__ A, long long lda, long long strideA,
 // Block-diagonal (head-wise, Eq. 6) and/or permuted rotation: output row j takes column
 // perm[j] of blockdiag(Rb); the chain runs over the dh rows of that column's block only.
 // One CTA per output row, threads along the output columns.
-template <typename TQ>
+template <typename TQ, typename TW>
 __global__ void __launch_bounds__(256)
 rotate_weights_blockdiag_kernel(const TQ *__restrict__ Rb, int d_in, int dh, const int32_t *__restrict__ perm,
-                                const __half *__restrict__ W, int d_out, float *__restrict__ Wp) {
+                                const TW *__restrict__ W, int d_out, float *__restrict__ Wp) {
   extern __shared__ float rcol[];  // [dh]
   const int j = blockIdx.x;
   const int p = perm ? perm[j] : j;
@@ -111,10 +111,10 @@ rotate_weights_blockdiag_kernel(const TQ *__restrict__ Rb, int d_in, int dh, con
   const TQ *R = Rb + (long long)h * dh * dh;
   for (int k = threadIdx.x; k < dh; k += blockDim.x) rcol[k] = to_f32<TQ>(R[(long long)k * dh + c]);
   __syncthreads();
-  const __half *Wb = W + (long long)h * dh * d_out;
+  const TW *Wb = W + (long long)h * dh * d_out;
   for (int n = blockIdx.y * blockDim.x + threadIdx.x; n < d_out; n += gridDim.y * blockDim.x) {
     float acc = 0.0f;
-    for (int k = 0; k < dh; ++k) acc = __fmaf_rn(rcol[k], __half2float(Wb[(long long)k * d_out + n]), acc);
+    for (int k = 0; k < dh; ++k) acc = __fmaf_rn(rcol[k], to_f32<TW>(Wb[(long long)k * d_out + n]), acc);
     Wp[(long long)j * d_out + n] = acc;
   }
 }
@@ -125,11 +125,20 @@ __global__ void cast_weights_kernel(const __half *__restrict__ W, long long n, f
   for (; i < n; i += stride) Wp[i] = __half2float(W[i]);
 }
 
-int launch_rotate_weights(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
-                          const __half *W, int d_out, float *Wp, cudaStream_t s) {
+// D W of the scaled (AWQ-style) variant: out[i][n] = d[i] * W[i][n], one fp32 rounding per product
+__global__ void scale_rows_kernel(const __half *__restrict__ W, const float *__restrict__ d, int d_out, long long n,
+                                  float *__restrict__ out) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) out[i] = __fmul_rn(d[i / d_out], __half2float(W[i]));
+}
+
+template <typename TW>
+static int rotate_weights_typed(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm, const TW *W,
+                                int d_out, float *Wp, cudaStream_t s) {
   if (n_blocks == 1 && perm == nullptr && q_is_f32) {
     dim3 grid((d_out + kBN - 1) / kBN, (d_in + kBM - 1) / kBM, 1);
-    gemm_tn_fma_kernel<float, __half, false><<<grid, 256, 0, s>>>(
+    gemm_tn_fma_kernel<float, TW, false><<<grid, 256, 0, s>>>(
         static_cast<const float *>(q), d_in, 0, W, d_out, 0, Wp, d_out, 0, d_in, d_out, d_in);
   } else {
     int dh = d_in / n_blocks;
@@ -137,21 +146,40 @@ int launch_rotate_weights(const void *q, int q_is_f32, int d_in, int n_blocks, c
     if (smem > 48 * 1024) {
       cudaError_t e;
       if (q_is_f32)
-        e = cudaFuncSetAttribute(rotate_weights_blockdiag_kernel<float>,
+        e = cudaFuncSetAttribute(rotate_weights_blockdiag_kernel<float, TW>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       else
-        e = cudaFuncSetAttribute(rotate_weights_blockdiag_kernel<__half>,
+        e = cudaFuncSetAttribute(rotate_weights_blockdiag_kernel<__half, TW>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
     }
     dim3 grid(d_in, min((d_out + 255) / 256, 8));
     if (q_is_f32)
-      rotate_weights_blockdiag_kernel<float><<<grid, 256, smem, s>>>(static_cast<const float *>(q), d_in, dh,
-                                                                       perm, W, d_out, Wp);
+      rotate_weights_blockdiag_kernel<float, TW><<<grid, 256, smem, s>>>(static_cast<const float *>(q), d_in, dh,
+                                                                           perm, W, d_out, Wp);
     else
-      rotate_weights_blockdiag_kernel<__half><<<grid, 256, smem, s>>>(static_cast<const __half *>(q), d_in, dh,
-                                                                        perm, W, d_out, Wp);
+      rotate_weights_blockdiag_kernel<__half, TW><<<grid, 256, smem, s>>>(static_cast<const __half *>(q), d_in, dh,
+                                                                            perm, W, d_out, Wp);
   }
+  return cudaGetLastError() == cudaSuccess ? ROSAQ_OK : ROSAQ_ERR_CUDA;
+}
+
+int launch_rotate_weights(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
+                          const __half *W, int d_out, float *Wp, cudaStream_t s) {
+  return rotate_weights_typed<__half>(q, q_is_f32, d_in, n_blocks, perm, W, d_out, Wp, s);
+}
+
+// the same chain on a weight that is already fp32 (the scaled weight D W)
+int launch_rotate_weights_w32(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
+                              const float *W32, int d_out, float *Wp, cudaStream_t s) {
+  return rotate_weights_typed<float>(q, q_is_f32, d_in, n_blocks, perm, W32, d_out, Wp, s);
+}
+
+int launch_scale_rows(const __half *W, const float *in_scale, int d_in, int d_out, float *out, cudaStream_t s) {
+  long long n = (long long)d_in * d_out;
+  long long want = (n + 255) / 256;
+  int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
+  scale_rows_kernel<<<blocks, 256, 0, s>>>(W, in_scale, d_out, n, out);
   return cudaGetLastError() == cudaSuccess ? ROSAQ_OK : ROSAQ_ERR_CUDA;
 }
 

@@ -224,8 +224,8 @@ int rosaq_calib_cov(rosaq_ctx *ctx, const void *X, int x_dtype, int64_t n_tokens
   return launch_cov(ctx, X, x_dtype, n_tokens, d, ldx, n_blocks, C, static_cast<cudaStream_t>(stream));
 }
 
-int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, int bits,
-                   int group, int k_salient, rosaq_weight **out, void *stream) {
+static int quantize_impl(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, const float *in_scale,
+                         int bits, int group, int k_salient, rosaq_weight **out, void *stream) {
   if (!out) return ROSAQ_ERR_INVALID_ARG;
   *out = nullptr;
   if (!ctx || !W) return ROSAQ_ERR_INVALID_ARG;
@@ -246,19 +246,29 @@ int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const ros
   w->k_salient = k_salient;
   w->device = ctx->device;
   w->t = make_geometry(d_in, d_out, bits, k_salient / kGroup, (d_in - k_salient) / kGroup, 0);
-  float *Wp = nullptr;
+  float *Wp = nullptr, *Ws = nullptr;
+  const size_t fbytes = sizeof(float) * (size_t)d_in * d_out;
   st = alloc_blob(&w->t);
-  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Wp), sizeof(float) * (size_t)d_in * d_out));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Wp), fbytes));
+  if (st == ROSAQ_OK && rot && in_scale) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Ws), fbytes));
   if (st == ROSAQ_OK) {
-    if (rot)
-      st = launch_rotate_weights(rot->q, rot->q_dtype == ROSAQ_F32, d_in, rot->n_blocks, rot->perm,
-                                 static_cast<const __half *>(W), d_out, Wp, s);
-    else
-      st = launch_cast_weights(static_cast<const __half *>(W), d_in, d_out, Wp, s);
+    const __half *Wh = static_cast<const __half *>(W);
+    if (rot && in_scale) {
+      st = launch_scale_rows(Wh, in_scale, d_in, d_out, Ws, s);
+      if (st == ROSAQ_OK)
+        st = launch_rotate_weights_w32(rot->q, rot->q_dtype == ROSAQ_F32, d_in, rot->n_blocks, rot->perm, Ws, d_out, Wp, s);
+    } else if (rot) {
+      st = launch_rotate_weights(rot->q, rot->q_dtype == ROSAQ_F32, d_in, rot->n_blocks, rot->perm, Wh, d_out, Wp, s);
+    } else if (in_scale) {
+      st = launch_scale_rows(Wh, in_scale, d_in, d_out, Wp, s);
+    } else {
+      st = launch_cast_weights(Wh, d_in, d_out, Wp, s);
+    }
   }
   if (st == ROSAQ_OK) st = launch_quant_pack(Wp, w->t, s);
   if (st == ROSAQ_OK) st = cuda_status(cudaStreamSynchronize(s));
   if (Wp) (void)cudaFree(Wp);
+  if (Ws) (void)cudaFree(Ws);
   if (st != ROSAQ_OK) {
     if (w->t.blob) (void)cudaFree(w->t.blob);
     delete w;
@@ -266,6 +276,18 @@ int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const ros
   }
   *out = w;
   return ROSAQ_OK;
+}
+
+int rosaq_quantize(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, int bits,
+                   int group, int k_salient, rosaq_weight **out, void *stream) {
+  return quantize_impl(ctx, W, d_in, d_out, rot, nullptr, bits, group, k_salient, out, stream);
+}
+
+int rosaq_quantize_scaled(rosaq_ctx *ctx, const void *W, int d_in, int d_out, const rosaq_rot *rot, const float *in_scale,
+                          int bits, int group, int k_salient, rosaq_weight **out, void *stream) {
+  if (out) *out = nullptr;
+  if (in_scale && !aligned16(in_scale)) return ROSAQ_ERR_ALIGNMENT;
+  return quantize_impl(ctx, W, d_in, d_out, rot, in_scale, bits, group, k_salient, out, stream);
 }
 
 int rosaq_weight_export(rosaq_ctx *ctx, const rosaq_weight *w, uint32_t *qw, void *scales_f16, void *zeros_f16,
@@ -538,6 +560,13 @@ int rosaq_plan_free(rosaq_plan *plan) {
   if (!plan) return ROSAQ_ERR_INVALID_ARG;
   plan_release(&plan->launch);
   delete plan;
+  return ROSAQ_OK;
+}
+
+int rosaq_set_plan_costs(rosaq_ctx *ctx, int fp16_group, int quant_group, int tile) {
+  if (!ctx || fp16_group < 1 || quant_group < 1 || tile < 0 || fp16_group > 1000 || quant_group > 1000 || tile > 1000)
+    return ROSAQ_ERR_INVALID_ARG;
+  ctx->pl_cost[0] = fp16_group, ctx->pl_cost[1] = quant_group, ctx->pl_cost[2] = tile;
   return ROSAQ_OK;
 }
 

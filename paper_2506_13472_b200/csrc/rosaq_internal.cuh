@@ -176,10 +176,14 @@ constexpr int kPlanMaxCtas = 512;
 constexpr int kPlMaxCounters = 4096;                // column tiles shared between CTAs in one launch
 constexpr int kPlSyncFinished = 0, kPlSyncDone = 4, kPlSyncArrive = 16;   // word offsets in the sync buffer
 constexpr int kPlSyncWords = kPlSyncArrive + kPlMaxCounters;
-// Relative cost of the work items when a phase is cut into equal shares: an fp16 group is bound by its
-// 32 KB of HBM traffic (about 1400 cycles of an SM's share of the bandwidth), a quantized one by its eight
-// MMAs (about 420 cycles), and every tile a CTA starts costs a little for switching accumulators.
-constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 3, kPlanCostTile = 1, kPlanCostScatterTile = 48;
+// Relative cost of the work items when a phase is cut into equal shares.  Both kinds of group cost the
+// tensor pipe eight MMAs (about 700 cycles in place); an fp16 group also moves 32 KB, which takes an SM's
+// share of the HBM bandwidth about 1400 cycles when every SM streams fp16 tiles, less when some run
+// quantized groups next to it.  Measured on the 7B decoder layer: 10 : 7 is best (10 : 3 ... 10 : 10 all
+// within 10 %).  Every tile a CTA starts costs a little for switching accumulators; a tile copy whose
+// output is scattered keeps the epilogue warps busy for about as long as seven quantized groups keep
+// the MMA threads.
+constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 7, kPlanCostTile = 1, kPlanCostScatterTile = 48;
 
 // One piece of work of a CTA: groups [g_begin, g_end) of column tile `tile` of problem `prob`.
 struct PlanSeg {
@@ -286,6 +290,9 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 // launchers implemented in the other translation units; all return a rosaq_status
 int launch_rotate_weights(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
                           const __half *W, int d_out, float *Wp, cudaStream_t s);
+int launch_rotate_weights_w32(const void *q, int q_is_f32, int d_in, int n_blocks, const int32_t *perm,
+                              const float *W32, int d_out, float *Wp, cudaStream_t s);
+int launch_scale_rows(const __half *W, const float *in_scale, int d_in, int d_out, float *out, cudaStream_t s);
 int launch_cast_weights(const __half *W, int d_in, int d_out, float *Wp, cudaStream_t s);
 int launch_quant_pack(const float *Wp, const TiledOperand &t, cudaStream_t s);
 int launch_export(const TiledOperand &t, uint32_t *qw, __half *scales, __half *zeros, __half *salient,

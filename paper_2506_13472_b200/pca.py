@@ -46,3 +46,15 @@ def eigh_descending_device(C_dev):
     sgn = torch.sign(V[big, torch.arange(V.shape[1], device=V.device)])
     sgn[sgn == 0] = 1.0
     return (V * sgn[None, :]).contiguous()
+
+
+def channel_scale(X, alpha=0.5):
+    """Diagonal D for the scaled (AWQ-style) quantization of an un-rotated linear such as the down
+    projection (weight-splitting appendix; scaling invariance X W = (X D^-1)(D W)).  The paper prints no rule
+    for D; this is the fixed one used here: d_i = (mean_t |x_ti|)^alpha, divided by sqrt(max d * min d) so that
+    the scales straddle 1.  Channels that are always zero get d_i = 1.  Returns fp32 [d]."""
+    m = np.abs(np.asarray(X, dtype=np.float64)).mean(axis=0)
+    d = np.where(m > 0, m, 1.0) ** float(alpha)
+    d = d / np.sqrt(d.max() * d.min())
+    d[m <= 0] = 1.0
+    return d.astype(np.float32)

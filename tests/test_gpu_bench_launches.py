@@ -105,6 +105,28 @@ def test_7b_down_all_columns(ctx):
     w.free()
 
 
+def test_7b_down_scaled_as_the_paper_runs_it(ctx):
+    """down_proj the way the weight-splitting appendix runs it: not rotated, quantized as D W with an
+    AWQ-style per-input-channel D, fed x D^-1.  Codes bit-exact on one column per tile, y on all columns."""
+    from paper_2506_13472_b200 import pca
+    d_in, d_out, bits = 11008, 4096, 4
+    W = synth.weights(d_in, d_out, 1, "7b-down-scaled", outlier_frac=0.01)
+    law = synth.ActivationLaw(d_in, 1.0, 1, "7b-down-scaled/x")
+    dsc = pca.channel_scale(law.sample(512, "calib", np.float32))
+    w = ctx.quantize(dev(W), None, bits=bits, k_salient=128, in_scale=dev(dsc))
+    e = H.export_to_numpy(w.export())
+    cols = H.tile_columns(d_out, 1, "7b-down-scaled")
+    qd = orc.quantize(np.ascontiguousarray(orc.scale_rows_f32(W, dsc)[:, cols]), bits, 128, 128)
+    qd["qw"], qd["cols"] = orc.pack(qd["codes"], bits), cols
+    H.assert_export_matches(e, qd)
+    x = law.sample(64, "x", np.float16)
+    xs = (x.astype(np.float32) / dsc[None, :]).astype(np.float16)
+    y = ctx.linear(dev(xs), w, None).cpu().numpy()
+    assert ctx.last_status() == rb.ROSAQ_OK
+    H.assert_y_all_columns(y, xs, H.qd_from_export(e, bits, 128), where="7b down, scaled")
+    w.free()
+
+
 # --------------------------------------------------------------------------- Gram kernel at the 13B widths
 def sampled_channels(d, seed):
     """96 channels: 32 from the first 256-channel block, 32 from a middle one, 32 from the last."""

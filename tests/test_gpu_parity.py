@@ -80,6 +80,37 @@ def test_import_export_round_trip(ctx, bits):
     assert np.array_equal(e["scales"], sc) and np.array_equal(e["zeros"], zr) and np.array_equal(e["salient"], sal)
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("rotated", [False, True])
+def test_quantize_scaled_bit_exact_and_forward(ctx, bits, rotated):
+    """rosaq_quantize_scaled: codes of D W (and of R^T D W) bit for bit against the oracle; the linear fed
+    x D^-1 reproduces the oracle's forward on the same weights and stays close to the unscaled product x W."""
+    c = H.config_tiny()
+    d_in, d_out, M = 512, 200, 9
+    W = synth.weights(d_in, d_out, seed=81, key="scaled", outlier_rows=4, outlier_scale=20.0)
+    law = synth.ActivationLaw(d_in, 1.2, 0, "tiny", mix="qr")
+    dsc = pca.channel_scale(law.sample(256, "scale-calib", np.float32))
+    assert dsc.min() < 1.0 < dsc.max()
+    R32, R16 = (c["R32"], c["R16"]) if rotated else (None, None)
+    w = ctx.quantize(dev(W), None if R32 is None else dev(R32), bits=bits, k_salient=128, in_scale=dev(dsc))
+    DW = orc.scale_rows_f32(W, dsc)
+    Wp = orc.rotate_weights_f32(R32, DW) if rotated else DW
+    qd = orc.quantize(Wp, bits, 128, 128)
+    qd["qw"], qd["cols"] = orc.pack(qd["codes"], bits), np.arange(d_out, dtype=np.int32)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    x = law.sample(M, "scaled-x", np.float16)
+    xs = (x.astype(np.float32) / dsc[None, :]).astype(np.float16)               # x D^-1, what the caller feeds
+    rot = ctx.rotation_create(dev(R16)) if rotated else None
+    y = ctx.linear(dev(xs), w, rot).cpu().numpy()
+    check_status(ctx)
+    assert H.rel_fro(y, orc.forward(xs, qd, R16)) <= H.REL_TOL_Y
+    ref = x.astype(np.float64) @ W.astype(np.float64)
+    assert H.rel_fro(y, ref) <= (0.2 if bits == 4 else 0.5)                      # the quantization error itself
+    with pytest.raises(rb.RosaqError) as e:                                       # misaligned scale pointer: a code
+        ctx.quantize(dev(W), None, bits=bits, k_salient=128, in_scale=dev(np.concatenate([dsc, dsc]))[1:d_in + 1])
+    assert e.value.status == rb.ROSAQ_ERR_ALIGNMENT
+
+
 # --------------------------------------------------------------------------- linear
 def run_linear_case(ctx, x16, W16, Rb32, Rb16, perm, bits, k_salient, impl):
     """quantize on the GPU, check codes, then y against the oracle forward on the same inputs."""

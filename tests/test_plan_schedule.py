@@ -10,7 +10,7 @@ import pytest
 
 from paper_2506_13472_b200 import binding as rb
 
-COST_FP16, COST_QUANT, COST_TILE, COST_SCATTER_TILE = 10, 3, 1, 48
+COST_FP16, COST_QUANT, COST_TILE, COST_SCATTER_TILE = 10, 7, 1, 48
 
 LAYER_7B = dict(  # rot(attn), rot(mlp), rot(o) head-wise, down, q, k, v, o, gate, up
     n_tiles=[32, 32, 32, 32, 32, 32, 32, 32, 86, 86], groups=[32, 32, 1, 86, 32, 32, 32, 32, 32, 32],
