@@ -108,6 +108,38 @@ def assemble_headwise_rotation(lams, Vs):
     return np.ascontiguousarray(Vs, np.float64), perm
 
 
+def assemble_headwise_rotation_per_head(lams, Vs, per_head=32):
+    """The paper's own W_O layout (weight-splitting appendix): each head keeps its `per_head` largest-eigenvalue
+    directions salient.  lams [H][dh] descending per head.  Column j of R is column perm[j] of
+    blockdiag(V_1..V_H): the salient directions of head 0, 1, ... first, then every head's remaining ones.
+    Returns (Rb, perm, K = H * per_head)."""
+    lams = np.asarray(lams, np.float64)
+    H, dh = lams.shape
+    assert np.all(np.diff(lams, axis=1) <= 0)
+    perm = [h * dh + i for h in range(H) for i in range(per_head)]
+    perm += [h * dh + i for h in range(H) for i in range(per_head, dh)]
+    return np.ascontiguousarray(Vs, np.float64), np.asarray(perm, np.int32), H * per_head
+
+
+def selection_order(lam, k_salient, mode, rng=None):
+    """Salient-selection ablation: the column order that puts the chosen k_salient directions first.  lam is
+    the descending eigenvalue vector (only its length and order are used)."""
+    d = len(lam)
+    order = list(range(d))
+    if mode == "top":
+        sel = order[:k_salient]
+    elif mode == "bottom":
+        sel = order[d - k_salient:]
+    elif mode == "random":
+        sel = sorted(rng.choice(d, size=k_salient, replace=False).tolist())
+    elif mode == "top_bottom":
+        sel = order[:k_salient // 2] + order[d - (k_salient - k_salient // 2):]
+    else:
+        raise ValueError(mode)
+    chosen = set(sel)
+    return np.asarray(sel + [i for i in order if i not in chosen], np.int32)
+
+
 def dense_from_blocks(Rb, perm=None):
     """The d x d matrix R that (Rb, perm) stands for."""
     Rb = np.asarray(Rb)

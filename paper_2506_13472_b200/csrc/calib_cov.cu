@@ -19,6 +19,8 @@
 // Every wait is bounded (ROSAQ_ERR_TIMEOUT through the context's status word).
 #include <cuda.h>
 
+#include <mutex>
+
 #include "rosaq_internal.cuh"
 
 namespace rosaq {
@@ -612,18 +614,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn cov_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static const EncodeTiledFn fn = [] {                       // initialised once, thread-safe
     void *sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-    else
-      (void)cudaGetLastError();
-  }
+      return reinterpret_cast<EncodeTiledFn>(sym);
+    (void)cudaGetLastError();
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 
@@ -675,6 +674,8 @@ int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tok
   static bool attr_done_all[64] = {};                    // function attributes are per device
   if (ctx->device < 0 || ctx->device >= 64) return ROSAQ_ERR_INVALID_ARG;
   bool &attr_done = attr_done_all[ctx->device];
+  static std::mutex attr_mutex;                          // contexts of several host threads share this cache
+  std::lock_guard<std::mutex> attr_lock(attr_mutex);
   if (!attr_done) {
     if (cudaFuncSetAttribute(cov_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       (void)cudaGetLastError();

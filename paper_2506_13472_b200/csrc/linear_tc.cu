@@ -22,6 +22,8 @@
 // status word, stops issuing work, still joins the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "linear_common.cuh"
 
 namespace rosaq {
@@ -738,18 +740,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static const EncodeTiledFn fn = [] {                       // initialised once, thread-safe
     void *sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-    else
-      (void)cudaGetLastError();
-  }
+      return reinterpret_cast<EncodeTiledFn>(sym);
+    (void)cudaGetLastError();
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 
@@ -799,23 +798,11 @@ bool sk_bounds(int T, int G, int g_fp16, int P, int *bounds) {
 
 }  // namespace
 
-// Tuning overrides, read from the environment once per process:
-//   ROSAQ_TC_SPLITS  number of K splits (1..8) instead of the heuristic
-//   ROSAQ_TC_PDL     0 = launch without programmatic stream serialization
-//   ROSAQ_TC_SK      0 = never use the stream-K variant; n > 1 = use it when CTAs <= n x column tiles
-struct TcOverrides {
-  int splits, pdl, sk;
-};
-static const TcOverrides &tc_overrides() {
-  static const TcOverrides o = [] {
-    auto read = [](const char *name, int dflt) {
-      const char *v = getenv(name);
-      return v && *v ? atoi(v) : dflt;
-    };
-    return TcOverrides{read("ROSAQ_TC_SPLITS", 0), read("ROSAQ_TC_PDL", 1), read("ROSAQ_TC_SK", 2)};
-  }();
-  return o;
-}
+// Launch policy of the per-call kernels (fixed; measured on the 7B / 13B shapes):
+//   kUsePdl      launches are chained with programmatic stream serialization
+//   kSkTileRatio the equal-share variant is used when CTAs <= kSkTileRatio x column tiles
+constexpr bool kUsePdl = true;
+constexpr int kSkTileRatio = 2;
 
 static int launch_linear_sk(const rosaq_ctx *ctx, const __half *x, long long ldx, const TiledOperand &t, const SkParams &q,
                             int P, cudaStream_t s) {
@@ -829,6 +816,8 @@ static int launch_linear_sk(const rosaq_ctx *ctx, const __half *x, long long ldx
   static size_t attr_smem_all[kMaxDevices][2] = {};       // function attributes are per device
   if (ctx->device < 0 || ctx->device >= kMaxDevices) return ROSAQ_ERR_INVALID_ARG;
   size_t *attr_smem = attr_smem_all[ctx->device];
+  static std::mutex attr_mutex;                           // contexts of several host threads share these caches
+  std::lock_guard<std::mutex> attr_lock(attr_mutex);
   if (attr_smem[int3 ? 1 : 0] < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -844,7 +833,7 @@ static int launch_linear_sk(const rosaq_ctx *ctx, const __half *x, long long ldx
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   int na = 0;
-  if (tc_overrides().pdl) {
+  if (kUsePdl) {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
@@ -919,9 +908,9 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   // is shared by two or three CTAs at most (its finisher reads the others' partial tiles one after the
   // other; measured at 64 tokens: 4096 -> 22016, 172 tiles, 23.4 us against 28.4 with cluster splits;
   // with 96 tiles 0.7 us slower, with 86 tiles 2.2 us slower)
-  if (ctx->impl == 0 && !pair && m_tiles == 1 && p.MT <= kSkTokens && ctx->sk_partials && tc_overrides().sk > 0) {
+  if (ctx->impl == 0 && !pair && m_tiles == 1 && p.MT <= kSkTokens && ctx->sk_partials) {
     const int P = ctx->sk_ctas < 2 * ctx->sm_count ? ctx->sk_ctas : 2 * ctx->sm_count;
-    if (n_tiles_all <= P && n_tiles_all <= kSkCounterInts && (long long)n_tiles_all * tc_overrides().sk >= P) {
+    if (n_tiles_all <= P && n_tiles_all <= kSkCounterInts && (long long)n_tiles_all * kSkTileRatio >= P) {
       SkParams q{};
       if (sk_bounds(n_tiles_all, G, t.g_fp16, P, q.bounds)) {
         q.n_prob = n;
@@ -959,8 +948,6 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   const int auto_cap = pair ? max_splits : 6;
   S = S < 1 ? 1 : (S > auto_cap ? auto_cap : S);
   if (S > G) S = G;
-  const int forced = tc_overrides().splits;
-  if (forced >= 1 && forced <= max_splits && forced <= G) S = forced;
   p.S = S;
   {
     // bound sp is the first group whose
@@ -1003,6 +990,8 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
   if (ctx->device < 0 || ctx->device >= kMaxDevices) return ROSAQ_ERR_INVALID_ARG;
   size_t *attr_smem = attr_smem_all[ctx->device];
   const int ki = (int3 ? 1 : 0) + (pair ? 2 : 0);
+  static std::mutex attr_mutex;                          // contexts of several host threads share these caches
+  std::lock_guard<std::mutex> attr_lock(attr_mutex);
   if (attr_smem[ki] < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -1025,7 +1014,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
     attr[na].val.clusterDim.z = 1;
     ++na;
   }
-  if (tc_overrides().pdl) {
+  if (kUsePdl) {
     // programmatic dependent launch: this kernel may start while the previous kernel of the stream is
     // still running; it touches x and y only after griddepcontrol.wait
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -424,9 +424,31 @@ __global__ void invert_perm_kernel(const int32_t *__restrict__ perm, int d, int3
   }
 }
 
-int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, cudaStream_t s) {
+// bad[0] = 1 when perm is not a permutation of 0..d-1: an entry out of range, or (inv still -1 somewhere
+// after the scatter above) a value that never occurs, i.e. another one occurs twice
+__global__ void check_perm_kernel(const int32_t *__restrict__ perm, const int32_t *__restrict__ inv, int d,
+                                  int *__restrict__ bad) {
+  int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < d && (perm[j] < 0 || perm[j] >= d || inv[j] < 0)) atomicExch(bad, 1);
+}
+
+// inv[perm[j]] = j.  Synchronizes the stream; ROSAQ_ERR_INVALID_ARG when perm is not a permutation (nothing
+// that indexes with it has been launched then).  `bad` is a device word owned by the caller.
+int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, int *bad, cudaStream_t s) {
+  if (cudaMemsetAsync(inv, 0xff, sizeof(int32_t) * (size_t)d, s) != cudaSuccess ||
+      cudaMemsetAsync(bad, 0, sizeof(int), s) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
   invert_perm_kernel<<<(d + 255) / 256, 256, 0, s>>>(perm, d, inv);
-  return cudaGetLastError() == cudaSuccess ? ROSAQ_OK : ROSAQ_ERR_CUDA;
+  check_perm_kernel<<<(d + 255) / 256, 256, 0, s>>>(perm, inv, d, bad);
+  int host = 0;
+  if (cudaGetLastError() != cudaSuccess || cudaMemcpyAsync(&host, bad, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
+  return host ? ROSAQ_ERR_INVALID_ARG : ROSAQ_OK;
 }
 
 }  // namespace rosaq

@@ -68,9 +68,17 @@ int run_gemm(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledO
   return launch_linear_tc(ctx, x, M, ldx, t, col_map, y, ldy, s);
 }
 
-// Up to 64 tokens the default implementation runs everything a call needs -- the rotation and the
-// linears that consume it -- as one persistent launch.
-bool use_plan(const rosaq_ctx *ctx, int M) { return ctx->impl == 0 && M <= 64; }
+// The persistent launch (rosaq_plan) pays off when a list is long: it saves a launch, a pipeline fill and a
+// drain per operation, but a list of one or two operations exposes its own fixed costs (the exchange of
+// shared tiles goes through L2 instead of a cluster's shared memory, and the phase after a rotation starts
+// only when the rotation's last tile is written).  Measured at 64 tokens, 4096 -> 4096 INT4: a GEMM stage
+// alone 15.9 us against 9.7 us on the per-call kernel; rotation + linear 30.5 us against 20.7 us as two
+// launches; the ten operations of a 7B decoder layer 66 us against 100 us as seven launches.  So the single
+// calls stay on the per-call kernels; implementation 4 routes them through the persistent launch.
+bool use_plan(const rosaq_ctx *ctx, int M, bool with_rotation) {
+  (void)with_rotation;
+  return M <= 64 && ctx->impl == 4;
+}
 
 int run_ops(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, cudaStream_t s) {
   PlanLaunch l;
@@ -129,8 +137,8 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->pl_partials = nullptr;
   ctx->pl_partial_bytes = 0;
   ctx->pl_sync = nullptr;
-  st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), sizeof(int)));
-  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, sizeof(int)));
+  st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 2 * sizeof(int)));   // [1]: scratch flag of argument checks
+  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, 2 * sizeof(int)));
   // the stream-K workspace is taken here, once, so that no linear call ever allocates for it
   if (st == ROSAQ_OK)
     st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->sk_partials), (size_t)ctx->sk_ctas * 2 * rosaq::kSkPartialBytes));
@@ -207,7 +215,7 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
   if (!ctx) return 0;
   int prev = ctx->impl;
-  if (impl >= 0 && impl <= 3) ctx->impl = impl;
+  if (impl >= 0 && impl <= 4) ctx->impl = impl;
   return prev;
 }
 
@@ -249,6 +257,13 @@ static int quantize_impl(rosaq_ctx *ctx, const void *W, int d_in, int d_out, con
   float *Wp = nullptr, *Ws = nullptr;
   const size_t fbytes = sizeof(float) * (size_t)d_in * d_out;
   st = alloc_blob(&w->t);
+  if (st == ROSAQ_OK && rot && rot->perm) {
+    // the rotate kernels index R and W with perm: reject anything that is not a permutation first
+    int32_t *inv = nullptr;
+    st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&inv), sizeof(int32_t) * (size_t)d_in));
+    if (st == ROSAQ_OK) st = launch_invert_perm(rot->perm, d_in, inv, ctx->d_status + 1, s);
+    if (inv) (void)cudaFree(inv);
+  }
   if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Wp), fbytes));
   if (st == ROSAQ_OK && rot && in_scale) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&Ws), fbytes));
   if (st == ROSAQ_OK) {
@@ -375,11 +390,13 @@ int rosaq_rotation_create(rosaq_ctx *ctx, const rosaq_rot *rot, rosaq_rotation *
   const int bg = dh / kGroup;
   r->t = make_geometry(rot->d, rot->d, 4, bg, 0, rot->n_blocks == 1 ? 0 : bg);
   int st = alloc_blob(&r->t);
-  if (st == ROSAQ_OK) st = launch_rotation_tiles(static_cast<const __half *>(rot->q), rot->d, rot->n_blocks, r->t, s);
   if (st == ROSAQ_OK && rot->perm) {
+    // checked first: the epilogues store through col_map, so a perm that is not a permutation is an error
+    // code here, never a stray write later
     st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&r->col_map), sizeof(int32_t) * rot->d));
-    if (st == ROSAQ_OK) st = launch_invert_perm(rot->perm, rot->d, r->col_map, s);
+    if (st == ROSAQ_OK) st = launch_invert_perm(rot->perm, rot->d, r->col_map, ctx->d_status + 1, s);
   }
+  if (st == ROSAQ_OK) st = launch_rotation_tiles(static_cast<const __half *>(rot->q), rot->d, rot->n_blocks, r->t, s);
   if (st == ROSAQ_OK) st = cuda_status(cudaStreamSynchronize(s));
   if (st != ROSAQ_OK) {
     if (r->t.blob) (void)cudaFree(r->t.blob);
@@ -417,7 +434,7 @@ int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
   if (st != ROSAQ_OK) return st;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return ROSAQ_ERR_CUDA;
-  if (use_plan(ctx, M)) {
+  if (use_plan(ctx, M, false)) {
     const PlanOp op{static_cast<const __half *>(x), ldx, -1, &r->t, r->col_map, static_cast<__half *>(x_rot), ldxr};
     return run_ops(ctx, M, 1, &op, static_cast<cudaStream_t>(stream));
   }
@@ -441,7 +458,7 @@ int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
     st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
     if (st != ROSAQ_OK) return st;
   }
-  if (use_plan(ctx, M)) {
+  if (use_plan(ctx, M, r != nullptr)) {
     // one launch: x . R into the workspace (phase 1), the GEMM stage on it (phase 2)
     PlanOp ops[2];
     int n = 0;
@@ -481,7 +498,7 @@ int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const 
     st = ensure_workspace(ctx, sizeof(__half) * (size_t)M * r->d, s);
     if (st != ROSAQ_OK) return st;
   }
-  if (use_plan(ctx, M)) {
+  if (use_plan(ctx, M, r != nullptr)) {
     PlanOp ops[5];
     int k = 0;
     if (r) ops[k++] = PlanOp{xin, ldx, -1, &r->t, r->col_map, static_cast<__half *>(ctx->ws), r->d};

@@ -15,7 +15,7 @@ namespace rosaq {
 // Tiled operand layout.
 //
 // A [d_in][d_out] matrix that the GEMM kernels stream is cut into tiles of 128 input
-// channels (one quantization group, Section 3: "a group consists of 128 channels") by
+// channels (one quantization group: group size 128, Section 3) by
 // 128 output columns.  All tiles of one column tile are contiguous, in input-channel
 // order, so that a CTA walking down K reads one linear stretch of memory; every tile is
 // a self-contained blob that one bulk copy brings into shared memory:
@@ -300,7 +300,7 @@ int launch_export(const TiledOperand &t, uint32_t *qw, __half *scales, __half *z
 int launch_import(const TiledOperand &t, const uint32_t *qw, const __half *scales, const __half *zeros,
                   const __half *salient, cudaStream_t s);
 int launch_rotation_tiles(const __half *q, int d, int n_blocks, const TiledOperand &t, cudaStream_t s);
-int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, cudaStream_t s);
+int launch_invert_perm(const int32_t *perm, int d, int32_t *inv, int *bad, cudaStream_t s);
 int launch_cov_fma(const void *X, int x_dtype, long long n_tokens, int d, long long ldx, int n_blocks, float *C,
                    cudaStream_t s);
 int launch_cov(const rosaq_ctx *ctx, const void *X, int x_dtype, long long n_tokens, int d, long long ldx,

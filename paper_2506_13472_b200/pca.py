@@ -58,3 +58,38 @@ def channel_scale(X, alpha=0.5):
     d = d / np.sqrt(d.max() * d.min())
     d[m <= 0] = 1.0
     return d.astype(np.float32)
+
+
+def headwise_rotation_per_head_salient(C_blocks, per_head=32):
+    """Head-wise PCA with the paper's own W_O layout (weight-splitting appendix): every head keeps its
+    `per_head` most principal directions in FP16, so K = H * per_head salient channels in all.  Column order
+    of R = blockdiag(R_1..R_H)[:, perm]: first the top `per_head` directions of head 0, of head 1, ...,
+    then the remaining directions head by head, each head's in descending eigenvalue order; the quantization
+    groups (128 channels) run over that concatenation.  Returns (Rb [H][dh][dh] fp64, perm int32, K)."""
+    lams, Rs = zip(*[eigh_descending(Cb) for Cb in np.asarray(C_blocks)])
+    H, dh = len(Rs), Rs[0].shape[0]
+    base = np.arange(H)[:, None] * dh
+    top = (base + np.arange(per_head)[None, :]).reshape(-1)
+    rest = (base + np.arange(per_head, dh)[None, :]).reshape(-1)
+    return np.ascontiguousarray(Rs), np.concatenate([top, rest]).astype(np.int32), H * per_head
+
+
+def selection_order(d, k_salient, mode, seed=0):
+    """Column orders for the salient-selection ablation (appendix on selecting salient channels): given
+    eigenvectors already in descending eigenvalue order, the permutation whose first k_salient columns are the
+    chosen ones -- 'top' (the method), 'bottom', 'random', 'top_bottom' (half from each end) -- followed by
+    the others in descending order.  Pass it as `perm` next to the dense R (n_blocks = 1)."""
+    idx = np.arange(d)
+    if mode == "top":
+        sel = idx[:k_salient]
+    elif mode == "bottom":
+        sel = idx[d - k_salient:]
+    elif mode == "random":
+        sel = np.sort(np.random.Generator(np.random.PCG64(seed)).choice(d, size=k_salient, replace=False))
+    elif mode == "top_bottom":
+        sel = np.concatenate([idx[:k_salient // 2], idx[d - (k_salient - k_salient // 2):]])
+    else:
+        raise ValueError(mode)
+    mask = np.ones(d, bool)
+    mask[sel] = False
+    return np.concatenate([sel, idx[mask]]).astype(np.int32)

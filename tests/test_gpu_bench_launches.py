@@ -60,6 +60,11 @@ def multi_case(ctx, d_in, widths, bits, Ms, seed, key, sigma=0.02, heavy_tail=Fa
         outs = ctx.linear_multi(xr, ws, None)
         again = ctx.linear_multi(xr, ws, None)
         fused = ctx.linear_multi(dev(x), ws, rot)                # rotation inside the call
+        ctx.set_linear_impl(4)                                   # ... and the whole call as one persistent launch
+        try:
+            one_launch = ctx.linear_multi(dev(x), ws, rot)
+        finally:
+            ctx.set_linear_impl(0)
         assert ctx.last_status() == rb.ROSAQ_OK
         xr_np = xr.cpu().numpy()
         _, xr_ref = orc.forward(x, dict(qds[0], salient=qds[0]["salient"][:, :8], scales=qds[0]["scales"][:, :8],
@@ -71,6 +76,7 @@ def multi_case(ctx, d_in, widths, bits, Ms, seed, key, sigma=0.02, heavy_tail=Fa
             assert np.array_equal(got.view(np.uint16), a.cpu().numpy().view(np.uint16))     # reproducible
             H.assert_y_all_columns(got, xr_np, qds[i], where=f"{key} M={M} weight {i}")
             H.assert_y_all_columns(f.cpu().numpy(), xr_np, qds[i], where=f"{key} fused M={M} weight {i}")
+            H.assert_y_all_columns(one_launch[i].cpu().numpy(), xr_np, qds[i], where=f"{key} one launch M={M} weight {i}")
     for w in ws:
         w.free()
     rot.free()

@@ -169,3 +169,56 @@ def test_layer_chain_replayed_from_a_graph_gives_the_bits_of_separate_calls(ctx)
             assert torch.equal(got.view(torch.int16), ref.view(torch.int16))
     for h in (wg, wu, wd, rot):
         h.free()
+
+
+@pytest.mark.parametrize("impl", [0, 4])
+def test_headwise_paper_layout_32_salient_per_head(ctx, impl):
+    """The paper's own o_proj layout (weight-splitting appendix): 32 heads x 128, every head keeps its 32 most
+    principal directions in FP16, K = 1024; the remaining channels are quantized in groups of 128 that run over
+    the heads' concatenated rests.  Same interface, another permutation.  INT4, M = 64."""
+    from paper_2506_13472_b200 import pca
+    heads, hd, d = 32, 128, 4096
+    law = synth.HeadwiseActivationLaw(heads, hd, 3, "hw-paper")
+    X = law.sample(2048, "calib", np.float16)
+    Cb = orc.cov(X, n_blocks=heads)
+    lams, Vs = zip(*[orc.eigh_jacobi(Cb[h]) for h in range(heads)])
+    Rb, perm, K = orc.assemble_headwise_rotation_per_head(np.array(lams), np.array(Vs), 32)
+    assert K == 1024
+    Rb_p, perm_p, K_p = pca.headwise_rotation_per_head_salient(Cb, 32)          # the product-side helper: same order
+    assert K_p == K and np.array_equal(perm_p, perm)
+    Rb32, Rb16 = Rb.astype(np.float32), Rb.astype(np.float16)
+    W = synth.weights(d, d, 3, "hw-paper", outlier_frac=0.01)
+    cols = synth.sample_columns(d, N_COLS, 3, "hw-paper")
+    w = ctx.quantize(dev(W), dev(Rb32), dev(perm), bits=4, k_salient=K)
+    qd = H.oracle_quantized(W, Rb32, perm, 4, K, cols=cols)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    rot = ctx.rotation_create(dev(Rb16), dev(perm))
+    x = law.sample(64, "x", np.float16)
+    ctx.set_linear_impl(impl)
+    try:
+        y = ctx.linear(dev(x), w, rot).cpu().numpy()
+    finally:
+        ctx.set_linear_impl(0)
+    assert ctx.last_status() == rb.ROSAQ_OK
+    assert H.rel_fro(y[:, cols], orc.forward(x, qd, Rb16, perm)) <= H.REL_TOL_Y
+
+
+@pytest.mark.parametrize("mode", ["bottom", "random", "top_bottom"])
+def test_salient_selection_variants_as_permutations(ctx, mode):
+    """The ablation's other choices of the FP16 channels (bottom / random / half-and-half): a column
+    permutation next to the dense R.  Codes bit-exact, y within the tolerance, on the tiny configuration."""
+    from paper_2506_13472_b200 import pca
+    c = H.config_tiny()
+    perm = pca.selection_order(c["d"], 128, mode, seed=7)
+    w = ctx.quantize(dev(c["W"]), dev(c["R32"]), dev(perm), bits=4, k_salient=128)
+    qd = H.oracle_quantized(c["W"], c["R32"], perm, 4, 128)
+    H.assert_export_matches(H.export_to_numpy(w.export()), qd)
+    rot = ctx.rotation_create(dev(c["R16"]), dev(perm))
+    for impl in (0, 4):
+        ctx.set_linear_impl(impl)
+        try:
+            y = ctx.linear(dev(c["x"]), w, rot).cpu().numpy()
+        finally:
+            ctx.set_linear_impl(0)
+        assert ctx.last_status() == rb.ROSAQ_OK
+        assert H.rel_fro(y, orc.forward(c["x"], qd, c["R16"], perm)) <= H.REL_TOL_Y

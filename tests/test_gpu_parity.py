@@ -131,26 +131,28 @@ def run_linear_case(ctx, x16, W16, Rb32, Rb16, perm, bits, k_salient, impl):
             # pre-rotated input through the GEMM stage alone gives the same y bits
             y2 = ctx.linear(dev(xr), w, None).cpu().numpy()
             assert np.array_equal(y2.view(np.uint16), y.view(np.uint16))
+            again = ctx.linear(dev(x16), w, rot).cpu().numpy()          # and so does a second run
+            assert np.array_equal(again.view(np.uint16), y.view(np.uint16))
         check_status(ctx)
     finally:
         ctx.set_linear_impl(0)
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 0, 4])
 @pytest.mark.parametrize("bits", [4, 3])
 def test_linear_tiny_config(ctx, bits, impl):
     c = H.config_tiny()
     run_linear_case(ctx, c["x"], c["W"], c["R32"], c["R16"], None, bits, 128, impl)
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 0, 4])
 @pytest.mark.parametrize("bits", [4, 3])
 def test_linear_headwise(ctx, bits, impl):
     c = H.config_headwise()
     run_linear_case(ctx, c["x"], c["W"], c["Rb32"], c["Rb16"], c["perm"], bits, 128, impl)
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 0, 4])
 @pytest.mark.parametrize("M,d_in,d_out,bits,k_salient", [
     (1, 256, 8, 4, 128), (3, 256, 136, 3, 0), (17, 384, 128, 4, 384), (64, 1024, 640, 4, 128),
     (130, 512, 256, 3, 128), (257, 256, 200, 4, 0)])
@@ -339,7 +341,58 @@ def test_argument_errors_are_codes_not_faults(ctx):
     assert ctx.last_status() == rb.ROSAQ_OK
 
 
+def test_a_perm_that_is_not_a_permutation_is_a_status_code(ctx):
+    """A duplicated or out-of-range entry in rot->perm would make the kernels index and store through
+    garbage: both calls that take a perm check it on the device first and return a code, launching nothing
+    that uses it."""
+    c = H.config_headwise()
+    d = c["heads"] * c["head_dim"]
+    for bad in (np.where(np.arange(d) == 5, c["perm"][6], c["perm"]).astype(np.int32),       # a value twice
+                np.where(np.arange(d) == 9, d, c["perm"]).astype(np.int32),                  # out of range
+                np.where(np.arange(d) == 0, -1, c["perm"]).astype(np.int32)):
+        with pytest.raises(rb.RosaqError) as e:
+            ctx.rotation_create(dev(c["Rb16"]), dev(bad))
+        assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+        with pytest.raises(rb.RosaqError) as e:
+            ctx.quantize(dev(c["W"]), dev(c["Rb32"]), dev(bad), bits=4, k_salient=128)
+        assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+    assert ctx.last_status() == rb.ROSAQ_OK
+    rot = ctx.rotation_create(dev(c["Rb16"]), dev(c["perm"]))                                  # the real one still works
+    rot.free()
+
+
 # --------------------------------------------------------------------------- bounded waits
+@pytest.mark.parametrize("impl,d_in,d_out", [(3, 1024, 512), (0, 1024, 150 * 128), (4, 1024, 512), (4, 512, 512)])
+def test_expired_waits_in_the_linear_kernels_leave_the_context_usable(ctx, impl, d_in, d_out):
+    """With the wait limit cut to one poll the linear kernels (cluster split-K, equal shares with the
+    workspace exchange, the persistent launch with and without a rotation) may give up anywhere: they must
+    return ROSAQ_OK or ROSAQ_ERR_TIMEOUT, never hang or fault, and afterwards -- status read, limit
+    restored -- the same call reproduces the earlier result bit for bit (no counter left behind)."""
+    W = synth.weights(d_in, d_out, seed=91, key=f"tw{d_in}x{d_out}", outlier_frac=0.01)
+    w = ctx.quantize(dev(W), None, bits=4, k_salient=128)
+    rot = ctx.rotation_create(dev(H.config_tiny()["R16"])) if d_in == 512 else None
+    x = dev(synth.rng_for(91, "x", d_in).standard_normal((64, d_in)).astype(np.float16))
+    ctx.set_linear_impl(impl)
+    try:
+        want = ctx.linear(x, w, rot).cpu().numpy()
+        assert ctx.last_status() == rb.ROSAQ_OK
+        old = ctx.set_wait_limit(1)
+        try:
+            for _ in range(3):
+                ctx.linear(x, w, rot)
+                assert ctx.last_status() in (rb.ROSAQ_OK, rb.ROSAQ_ERR_TIMEOUT)
+        finally:
+            ctx.set_wait_limit(old)
+        for _ in range(2):
+            got = ctx.linear(x, w, rot).cpu().numpy()
+            assert ctx.last_status() == rb.ROSAQ_OK
+            assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    finally:
+        ctx.set_linear_impl(0)
+    w.free()
+
+
+
 def test_expired_wait_is_reported_and_the_context_stays_usable(ctx):
     """Failure detection without a GPU fault: with the wait limit cut to one poll, a wait that cannot be
     satisfied in time (the Gram kernel's epilogue waiting for ~100 us of accumulation) gives up: the

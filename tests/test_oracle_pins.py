@@ -483,3 +483,54 @@ def test_scaled_then_rotated_chain_takes_the_fp32_scaled_weight():
     # and it is the same chain as the binary16 entry when the scaled weight happens to be the widened one
     assert np.array_equal(orc.rotate_weights_f32(R, W.astype(np.float32)).view(np.uint32),
                           orc.rotate_weights_f32(R, W).view(np.uint32))
+
+
+# --------------------------------------------------------------------------- W_O layout and selection ablation
+def test_per_head_salient_layout_is_a_permutation_and_keeps_eq1():
+    """32 salient directions per head (weight-splitting appendix): the column order is a permutation, its
+    first H * 32 entries are exactly each head's 32 largest-eigenvalue directions, and the rotated linear
+    with this R still equals x W in fp64 (Eq. 1 / Eq. 6)."""
+    rng = np.random.default_rng(41)
+    H, dh, d_out, M = 4, 128, 12, 3
+    lams = -np.sort(-rng.uniform(0.1, 5.0, (H, dh)), axis=1)
+    Vs = np.array([synth.orthogonal_qr(dh, rng) for _ in range(H)])
+    Rb, perm, K = orc.assemble_headwise_rotation_per_head(lams, Vs, 32)
+    assert K == 128 and sorted(perm.tolist()) == list(range(H * dh))
+    assert perm[:K].tolist() == [h * dh + i for h in range(H) for i in range(32)]
+    for h in range(H):                                   # every salient column is among its head's 32 largest
+        mine = [p % dh for p in perm[:K] if p // dh == h]
+        assert sorted(mine) == list(range(32)) and lams[h, 31] >= lams[h, 32]
+    W = rng.standard_normal((H * dh, d_out))
+    x = rng.standard_normal((M, H * dh))
+    R = orc.dense_from_blocks(Rb, perm)
+    assert np.abs(R.T @ R - np.eye(H * dh)).max() <= 1e-12
+    Wp = orc.rotate_weights_f64(Rb, W, perm)
+    ref = x @ W
+    assert np.linalg.norm((x @ R) @ Wp - ref) / np.linalg.norm(ref) <= 1e-10
+
+
+@pytest.mark.parametrize("mode", ["top", "bottom", "random", "top_bottom"])
+def test_selection_orders_are_permutations_with_the_named_salient_set(mode):
+    rng = np.random.default_rng(42)
+    d, K = 256, 128
+    lam = -np.sort(-rng.uniform(0.0, 1.0, d))
+    perm = orc.selection_order(lam, K, mode, rng)
+    assert sorted(perm.tolist()) == list(range(d))
+    sel = set(perm[:K].tolist())
+    if mode == "top":
+        assert perm.tolist() == list(range(d))
+    elif mode == "bottom":
+        assert sel == set(range(d - K, d))
+    elif mode == "top_bottom":
+        assert sel == set(range(K // 2)) | set(range(d - K // 2, d))
+    assert np.all(np.diff(perm[K:]) > 0)                 # the others stay in descending-eigenvalue order
+    V = synth.orthogonal_qr(d, rng)
+    W = rng.standard_normal((d, 7))
+    x = rng.standard_normal((2, d))
+    Wp = orc.rotate_weights_f64(V, W, perm)
+    ref = x @ W
+    assert np.linalg.norm((x @ V[:, perm]) @ Wp - ref) / np.linalg.norm(ref) <= 1e-10
+    # the product helper agrees with the oracle's index rule
+    from paper_2506_13472_b200 import pca
+    if mode != "random":
+        assert np.array_equal(pca.selection_order(d, K, mode), perm)
