@@ -23,7 +23,7 @@ EXPORTS = [
     "rosaq_weight_import", "rosaq_weight_free", "rosaq_weight_info", "rosaq_rotation_create",
     "rosaq_rotation_free", "rosaq_rotate", "rosaq_linear", "rosaq_linear_multi", "rosaq_linear_static",
     "rosaq_plan_equal_shares", "rosaq_plan_create", "rosaq_plan_run", "rosaq_plan_free", "rosaq_plan_ctas",
-    "rosaq_plan_schedule", "rosaq_set_plan_costs",
+    "rosaq_plan_schedule", "rosaq_set_plan_costs", "rosaq_set_plan_pairs",
 ]
 
 
@@ -87,6 +87,7 @@ def lib():
         L.rosaq_plan_free.argtypes = [C.c_void_p]
         L.rosaq_plan_ctas.argtypes = [C.c_void_p]
         L.rosaq_set_plan_costs.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
+        L.rosaq_set_plan_pairs.argtypes = [C.c_void_p, C.c_int]
         L.rosaq_plan_schedule.argtypes = [C.c_int] + [C.POINTER(C.c_int32)] * 5 + [C.c_int, C.POINTER(C.c_int32),
                                                                                   C.POINTER(C.c_int32), C.c_int]
         _lib = L
@@ -259,6 +260,9 @@ class Context:
 
     def set_plan_costs(self, fp16_group, quant_group, tile):
         _check(lib().rosaq_set_plan_costs(self._h, fp16_group, quant_group, tile), "rosaq_set_plan_costs")
+
+    def set_plan_pairs(self, enable):
+        return lib().rosaq_set_plan_pairs(self._h, 1 if enable else 0)
 
     def plan_ctas(self):
         n = lib().rosaq_plan_ctas(self._h)

@@ -67,7 +67,7 @@ struct PlProblem {
   __half *y;
   const int32_t *col_map;
   long long tile_stride, ldy;
-  int d_out, g_fp16, block_groups;
+  int d_out, n_tiles, g_fp16, block_groups;
   int dep;                    // problem whose output this one reads, or -1
   unsigned dep_target;        // finishing events that complete problem `dep`
   int signal;                 // some problem reads this one's output: count finishing events
@@ -163,16 +163,27 @@ __device__ __forceinline__ void epi_finish(uint32_t d_addr, bool both, int c_beg
       for (int i = 1; i < S; ++i) {
         const float *src = src0 + (long long)i * slot_floats + c0 * kTileN;
         float w[CH];
+        if (c0 + CH <= M) {
 #pragma unroll
-        for (int e = 0; e < CH; ++e) w[e] = c0 + e < M ? __ldcg(src + e * kTileN) : 0.f;
+          for (int e = 0; e < CH; ++e) w[e] = __ldcg(src + e * kTileN);
+        } else {
+#pragma unroll
+          for (int e = 0; e < CH; ++e) w[e] = c0 + e < M ? __ldcg(src + e * kTileN) : 0.f;
+        }
 #pragma unroll
         for (int e = 0; e < CH; ++e) acc[e] = __fadd_rn(acc[e], w[e]);
       }
     }
+    __half *yp = y_col + (long long)c0 * ldy;
+    if (n_ok && c0 >= t0 && c0 + CH <= t1) {                  // the usual case: the whole batch is written
 #pragma unroll
-    for (int e = 0; e < CH; ++e) {
-      const int mg = c0 + e;
-      if (n_ok && mg >= t0 && mg < t1) y_col[(long long)mg * ldy] = __float2half_rn(acc[e]);
+      for (int e = 0; e < CH; ++e, yp += ldy) *yp = __float2half_rn(acc[e]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < CH; ++e, yp += ldy) {
+        const int mg = c0 + e;
+        if (n_ok && mg >= t0 && mg < t1) *yp = __float2half_rn(acc[e]);
+      }
     }
   }
 }
@@ -183,19 +194,33 @@ __device__ __forceinline__ void epi_store_partial(uint32_t d_addr, bool both, in
   for (int c0 = c_begin; c0 < c_end && c0 < M; c0 += CH) {
     float acc[CH];
     epi_load_acc<CH>(d_addr, both, c0, acc);
+    float *dp = dst + c0 * kTileN;
+    if (c0 + CH <= M) {
 #pragma unroll
-    for (int e = 0; e < CH; ++e)
-      if (c0 + e < M) dst[(c0 + e) * kTileN] = acc[e];
+      for (int e = 0; e < CH; ++e) dp[e * kTileN] = acc[e];
+    } else {
+#pragma unroll
+      for (int e = 0; e < CH; ++e)
+        if (c0 + e < M) dp[e * kTileN] = acc[e];
+    }
   }
 }
 
-template <int kBits>
+// kPair: the CTAs of a cluster of two (ranks 0 and 1, adjacent SMs) run as a cta_group::2 pair on one
+// schedule entry: a piece is then the groups of TWO adjacent column tiles, rank r dequantises tile 2 t + r into
+// its own tensor memory and loads half of the token rows, and the leader (rank 0) issues one M = 256 MMA for
+// both.  An MMA instruction costs the same 55 cycles whether it covers 128 or 256 rows, so the pair needs
+// 222 cycles of each SM's tensor pipe per 128-channel group where a single CTA needs 440 -- less than the
+// 375 cycles the group's bytes take.  Barriers that both CTAs feed live in the leader; its commits are
+// multicast to both.
+template <int kBits, bool kPair>
 __global__ void __launch_bounds__(kPlThreads, 1)
 linear_plan_kernel(const __grid_constant__ PlParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int MT = p.MT;
-  const uint32_t x_slot_bytes = (uint32_t)MT * 256u;
+  const int MTL = kPair ? MT >> 1 : MT;                        // token rows this CTA keeps in shared memory
+  const uint32_t x_slot_bytes = (uint32_t)MTL * 256u;
   const uint32_t x_ring = base;
   const uint32_t w_ring = x_ring + kPlStages * x_slot_bytes;
   const uint32_t bars = w_ring + p.NW * kWSlotBytes;
@@ -210,9 +235,12 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
   volatile uint32_t *misc_ptr = reinterpret_cast<volatile uint32_t *>(gen + (misc - base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int cta = blockIdx.x;
+  const uint32_t rank = kPair ? (blockIdx.x & 1u) : 0u;        // position in the pair; 0 = leader
+  const bool is_lead = rank == 0;
+  const int cta = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // entry of the schedule
   const int s_begin = p.seg_begin[cta], s_end = p.seg_begin[cta + 1];
-  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit, false};
+  const Abort ab{reinterpret_cast<volatile int *>(misc_ptr + 1), p.status, p.wait_limit, kPair};
+  const int tile_mul = kPair ? 2 : 1;                          // this CTA's column tile of a piece: tile_mul * tile + rank
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.NW; ++i) {
@@ -220,12 +248,13 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       mbar_init(bar_w_empty + 8 * i, kTeamThreads);
     }
     for (int i = 0; i < kPlStages; ++i) {
-      mbar_init(bar_a_full + 8 * i, kTeamThreads + 1);         // + the activation copy
+      // a team's arrivals (per thread; in a pair per warp, from both CTAs) + the activation copy
+      mbar_init(bar_a_full + 8 * i, (kPair ? 2 * (kTeamThreads / 32) : kTeamThreads) + 1);
       mbar_init(bar_s_empty + 8 * i, 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_d_full + 8 * i, 2);                        // both issuers
-      mbar_init(bar_d_empty + 8 * i, kPlEpiThreads);
+      mbar_init(bar_d_empty + 8 * i, (kPair ? 2 : 1) * (kPlEpiThreads / 32));   // one arrival per epilogue warp
       mbar_init(bar_drain + 8 * i, 1);
     }
     misc_ptr[1] = 0;
@@ -233,9 +262,16 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 2) tmem_alloc<kPlTmemCols>(misc);
+  if (warp == 2) {
+    if (kPair) tmem_alloc_pair<kPlTmemCols>(misc);             // both CTAs of the pair, same warp index
+    else tmem_alloc<kPlTmemCols>(misc);
+  }
   tc_fence_before();
   __syncthreads();
+  if (kPair) {                                                 // the peer's barriers and tensor memory exist
+    cluster_arrive();
+    cluster_wait();
+  }
   tc_fence_after();
   const uint32_t tmem = misc_ptr[0];
   const uint32_t a_col0 = 4 * kPlTokens;
@@ -244,38 +280,58 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
   if (warp == 0) {
     // ---------------- weight-tile producer: streams every piece of every phase, waits for ring slots only
     if (lane == 0) {
+      // The ring is split into one sub-ring of NWT slots per dequantisation team (group j of the CTA's stream
+      // belongs to team j mod 4): a sub-ring has one consumer, which takes its slots in order, so a full /
+      // empty pair of barriers per slot is enough.  Positions of the four sub-rings: a byte each in idx4,
+      // a bit each in lap4; fills per team in fills4 (16 bits each, only looked at when giving up).
       const uint64_t pol = policy_evict_first();
-      int uc = 0;
-      Ring rw{0, 0};
+      const int NWT = p.NW >> 2;
+      uint32_t idx4 = 0, lap4 = 0;
+      unsigned long long fills4 = 0;
+      int j = 0;
       bool live = true;
       for (int si = s_begin; si < s_end && live && !ab.set(); ++si) {
         const PlanSeg s = load_seg(p.segs + si);
         const PlProblem &P = p.prob[s.prob];
-        const uint8_t *tile_base = P.blob + (long long)s.tile * P.tile_stride;
+        // (the second CTA of a pair on an odd last tile streams that tile again; its results are dropped)
+        int my_tile = tile_mul * s.tile + (int)rank;
+        if (my_tile >= P.n_tiles) my_tile = P.n_tiles - 1;
+        const uint8_t *tile_base = P.blob + (long long)my_tile * P.tile_stride;
         const int g_fp16 = P.g_fp16;
-        for (int g = s.g_begin; g < s.g_end && live; ++g) {
+        for (int g = s.g_begin; g < s.g_end && live; ++g, ++j) {
           const bool f16 = g < g_fp16;
           const uint8_t *src = tile_base + (f16 ? (long long)g * kFp16TileBytes
                                                 : (long long)g_fp16 * kFp16TileBytes + (long long)(g - g_fp16) * qbytes);
           const int nsub = f16 ? 4 : 1;
           const uint32_t bytes = f16 ? kFp16SubBytes : qbytes;
-          for (int sub = 0; sub < nsub; ++sub, ++uc, rw.advance(p.NW)) {
-            const int slot = rw.idx;
-            if (!ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u)) {
+          const int team = j & (kPlTeams - 1);
+          uint32_t idx = (idx4 >> (8 * team)) & 0xffu;
+          for (int sub = 0; sub < nsub; ++sub) {
+            const int slot = team * NWT + (int)idx;
+            if (!ab.wait_local(bar_w_empty + 8 * slot, ((lap4 >> team) & 1u) ^ 1u)) {
               live = false;
               break;
             }
             mbar_arrive_expect_tx(bar_w_full + 8 * slot, bytes);
             bulk_copy_g2s_hint(w_ring + slot * kWSlotBytes, src + (long long)sub * kFp16SubBytes, bytes,
                                bar_w_full + 8 * slot, pol);
+            fills4 += 1ull << (16 * team);
+            if (++idx == (uint32_t)NWT) {
+              idx = 0;
+              lap4 ^= 1u << team;
+            }
           }
+          idx4 = (idx4 & ~(0xffu << (8 * team))) | (idx << (8 * team));
         }
       }
       if (ab.set()) {  // let copies already in flight land before the CTA goes away
-        for (int back = 1; back <= p.NW && back <= uc; ++back) {
-          const int u = uc - back;
-          for (int it = 0; it < kDrainPolls; ++it)
-            if (mbar_try_wait(bar_w_full + 8 * (u % p.NW), (u / p.NW) & 1)) break;
+        for (int team = 0; team < kPlTeams; ++team) {
+          const int f = (int)((fills4 >> (16 * team)) & 0xffffu);     // (mod 65536: only the last NWT fills matter)
+          for (int back = 1; back <= NWT && back <= f; ++back) {
+            const int u = f - back;
+            for (int it = 0; it < kDrainPolls; ++it)
+              if (mbar_try_wait(bar_w_full + 8 * (team * NWT + u % NWT), (u / NWT) & 1)) break;
+          }
         }
       }
     }
@@ -299,7 +355,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
           }
         }
         // block-diagonal operand: a column tile only multiplies the channels of its own diagonal block
-        const int g_block0 = P.block_groups > 0 ? (s.tile / P.block_groups) * P.block_groups : 0;
+        const int g_block0 = P.block_groups > 0 ? ((tile_mul * s.tile + (int)rank) / P.block_groups) * P.block_groups : 0;
         const CUtensorMap *map = &p.xmap[s.prob];
         for (int g = s.g_begin; g < s.g_end; ++g, ++gc, rs.advance(kPlStages)) {
           const int slot = rs.idx;
@@ -308,15 +364,23 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
             break;
           }
           const int k0 = (g_block0 + g) * kGroup;
-          mbar_arrive_expect_tx(bar_a_full + 8 * slot, x_slot_bytes);
-          tma_load_3d(x_ring + slot * x_slot_bytes, map, bar_a_full + 8 * slot, 0, k0 >> 6);
+          if (kPair) {
+            // each CTA loads its half of the token rows; all bytes are counted on the leader's barrier
+            if (is_lead) mbar_arrive_expect_tx(bar_a_full + 8 * slot, 2 * x_slot_bytes);
+            tma_load_3d_pair(x_ring + slot * x_slot_bytes, map, map_to_rank(bar_a_full + 8 * slot, 0), (int)rank * MTL, k0 >> 6);
+          } else {
+            mbar_arrive_expect_tx(bar_a_full + 8 * slot, x_slot_bytes);
+            tma_load_3d(x_ring + slot * x_slot_bytes, map, bar_a_full + 8 * slot, 0, k0 >> 6);
+          }
         }
       }
-      if (ab.set()) {
+      // (in a pair the leader's barriers count the copies of both CTAs, and the peer stays until the cluster
+      // barrier at the end of the kernel, which the leader reaches after this drain)
+      if (ab.set() && is_lead) {
         for (int back = 1; back <= kPlStages && back <= gc; ++back) {
           const int u = gc - back;
           for (int it = 0; it < kDrainPolls; ++it)
-            if (mbar_try_wait(bar_a_full + 8 * (u % kPlStages), (u / kPlStages) & 1)) break;
+            if (ab.poll(bar_a_full + 8 * (u % kPlStages), (u / kPlStages) & 1)) break;
         }
       }
     }
@@ -325,11 +389,12 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
     // j mod 2 == i (operand buffers i and i + 2) and accumulates them into its own tile; per group one
     // wait, eight MMAs, one commit.  Every piece is committed by both (an issuer without a group in a
     // one-group piece arrives by hand), so the epilogue waits for one barrier.
-    if (lane == 0) {
+    if (lane == 0 && is_lead) {
       const int me = warp - 2;
-      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | (8u << 24);
+      // M = 128 output columns (256 for a pair), N = MT tokens
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | ((kPair ? 16u : 8u) << 24);
       const uint64_t desc0 = make_b_desc(x_ring);
-      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MT * 128) >> 4;
+      const uint32_t x_slot16 = x_slot_bytes >> 4, half16 = (uint32_t)(MTL * 128) >> 4;
       int nseg = 0, j = 0;
       bool live = true, issued = false;
       for (int si = s_begin; si < s_end && live; ++si, ++nseg) {
@@ -339,8 +404,10 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         tc_fence_after();
         const uint32_t d_tmem = tmem + (uint32_t)(2 * buf + me) * kPlTokens;
         uint32_t accumulate = 0;
-        for (int g = s.g_begin; g < s.g_end; ++g, ++j) {
-          if ((j & 1) != me) continue;
+        const int g_first = s.g_begin + ((me - j) & 1), j_base = j - s.g_begin;
+        j += s.g_end - s.g_begin;
+        for (int g = g_first; g < s.g_end; g += 2) {
+          const int j = j_base + g;
           const int st = j & (kPlStages - 1);
           if (!ab.wait(bar_a_full + 8 * st, (uint32_t)(j >> 2) & 1u)) {
             live = false;
@@ -348,61 +415,79 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
           }
           tc_fence_after();
           const uint64_t b0 = desc0 + (uint64_t)(st * x_slot16);
-          tc_mma8_ts(d_tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
-          tc_commit(bar_s_empty + 8 * st);
+          if (kPair) {
+            tc_mma8_ts_pair(d_tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+            tc_commit_mc(bar_s_empty + 8 * st, 3);             // frees the stage in both CTAs
+          } else {
+            tc_mma8_ts(d_tmem, tmem + a_col0 + st * 64, b0, b0 + (uint64_t)half16, idesc, accumulate);
+            tc_commit(bar_s_empty + 8 * st);
+          }
           accumulate = 1;
           issued = true;
         }
         if (!live) break;
-        if (accumulate) tc_commit(bar_d_full + 8 * buf);
-        else mbar_arrive(bar_d_full + 8 * buf);
+        if (kPair) {
+          if (accumulate) tc_commit_mc(bar_d_full + 8 * buf, 3);
+          else {
+            mbar_arrive_cluster(map_to_rank(bar_d_full + 8 * buf, 0));
+            mbar_arrive_cluster(map_to_rank(bar_d_full + 8 * buf, 1));
+          }
+        } else {
+          if (accumulate) tc_commit(bar_d_full + 8 * buf);
+          else mbar_arrive(bar_d_full + 8 * buf);
+        }
       }
       if (ab.set() && issued) {  // MMAs already issued must retire before the tensor memory is given back
-        tc_commit(bar_drain + 8 * me);
+        if (kPair) tc_commit_mc(bar_drain + 8 * me, 1);
+        else tc_commit(bar_drain + 8 * me);
         for (int it = 0; it < kDrainPolls; ++it)
-          if (mbar_try_wait(bar_drain + 8 * me, 0)) break;
+          if (ab.poll(bar_drain + 8 * me, 0)) break;
       }
     }
   } else if (warp >= kPlFirstDequantWarp && warp < kPlFirstEpiWarp) {
-    // ---------------- dequantisation: group j of the CTA goes to team and operand buffer j mod 4
+    // ---------------- dequantisation: group j of the CTA's stream goes to team and operand buffer j mod 4;
+    // a team walks over its own groups only and takes the slots of its own sub-ring in order
     const int quad = warp & 3;
     const int team = (warp - kPlFirstDequantWarp) >> 2;
     const int n = quad * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    Ring rw{0, 0}, rs{0, 0};
+    const int NWT = p.NW >> 2;
+    const uint32_t my_ring = w_ring + team * NWT * kWSlotBytes, my_full = bar_w_full + 8 * team * NWT,
+                   my_empty = bar_w_empty + 8 * team * NWT;
+    const uint32_t a_addr = lane_addr + a_col0 + team * 64;
+    const uint32_t my_s_empty = bar_s_empty + 8 * team, my_a_full = bar_a_full + 8 * team;
+    Ring rw{0, 0};
     bool ok = true;
-    int j = 0;
+    int j0 = 0;                                      // position of the piece's first group in the CTA's stream
     for (int si = s_begin; si < s_end && ok; ++si) {
       const PlanSeg s = load_seg(p.segs + si);
       const int g_fp16 = p.prob[s.prob].g_fp16;
-      for (int g = s.g_begin; g < s.g_end && ok; ++g, ++j, rs.advance(kPlStages)) {
+      for (int g = s.g_begin + ((team - j0) & (kPlTeams - 1)); g < s.g_end && ok; g += kPlTeams) {
         const bool f16 = g < g_fp16;
         const int nsub = f16 ? 4 : 1;
-        if ((j & (kPlTeams - 1)) != team) {
-          for (int sub = 0; sub < nsub; ++sub) rw.advance(p.NW);
-          continue;
-        }
-        const int st = rs.idx;
-        const uint32_t a_addr = lane_addr + a_col0 + st * 64;
-        bool got = ab.wait(bar_s_empty + 8 * st, rs.lap ^ 1u);
-        for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(p.NW)) {
-          const int slot = rw.idx;
-          // first see the slot's previous fill released (it may belong to another team, which can lag),
-          // then wait for the new one: a parity wait must not be a whole phase early
-          got = got && ab.wait_local(bar_w_empty + 8 * slot, rw.lap ^ 1u) && ab.wait_local(bar_w_full + 8 * slot, rw.lap);
-          got = __all_sync(0xffffffffu, got);
+        const uint32_t use = (uint32_t)(j0 + g - s.g_begin) >> 2;        // how often this team's buffer was used before
+        bool got = ab.wait(my_s_empty, (use & 1u) ^ 1u);
+        for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(NWT)) {
+          got = got && ab.wait_local(my_full + 8 * rw.idx, rw.lap);
+          got = __all_sync(0xffffffffu, got);        // the TMEM instructions below need the whole warp
           if (!got) {
             ok = false;
             break;
           }
           tc_fence_after();
-          dequant_unit<kBits>(f16, w_ring + slot * kWSlotBytes, n, a_addr, sub, bar_w_empty + 8 * slot);
+          dequant_unit<kBits>(f16, my_ring + rw.idx * kWSlotBytes, n, a_addr, sub, my_empty + 8 * rw.idx);
         }
         tc_wait_st();
         if (!ok) break;
         tc_fence_before();
-        mbar_arrive(bar_a_full + 8 * st);
+        if (kPair) {                                           // one arrival per warp, on the leader's barrier
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(map_to_rank(my_a_full, 0));
+        } else {
+          mbar_arrive(my_a_full);
+        }
       }
+      j0 += s.g_end - s.g_begin;
     }
   } else if (warp >= kPlFirstEpiWarp) {
     // ---------------- epilogue: one pass per piece.  Thread = (output column n of the tile = TMEM lane,
@@ -429,7 +514,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       if (!have_d) break;
       tc_fence_after();
       const uint32_t d_addr = lane_addr + (uint32_t)(2 * buf + first_acc) * kPlTokens;
-      const int n_glob = s.tile * kTileN + n;
+      const int n_glob = (tile_mul * s.tile + (int)rank) * kTileN + n;
       const bool n_ok = n_glob < P.d_out;
       const long long out_col = n_ok ? (P.col_map ? P.col_map[n_glob] : n_glob) : 0;
       __half *const y_out = P.y;
@@ -439,8 +524,10 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       // the only closer of a shared tile (it holds the tile's first groups) keeps its accumulator and adds
       // the other holders' partial tiles to it
       const bool keep = !sole && s.n_closers == 1 && s.closer_idx == 0;
-      unsigned *ctr = p.sync + kPlSyncArrive + s.counter;
-      const float *src0 = p.partials + (long long)s.slot0 * p.slot_floats + n;
+      // (the two CTAs of a pair exchange their own tiles: slots and counters are interleaved by rank)
+      unsigned *ctr = p.sync + kPlSyncArrive + tile_mul * s.counter + rank;
+      const long long slot_step = (long long)tile_mul * p.slot_floats;            // from one holder's slot to the next
+      const float *src0 = p.partials + ((long long)tile_mul * s.slot0 + rank) * p.slot_floats + n;
       if (keep) {
         if (lead) wait_counter(ab, ctr, (unsigned)(S - 1));
         epi_bar();
@@ -448,10 +535,14 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       }
       if (sole || keep) {
         const int t0 = s.tok_begin, t1 = s.tok_end < p.M ? s.tok_end : p.M;     // token rows this piece writes
-        if (wide) epi_finish<16>(d_addr, both, c_begin, c_end, keep, S, src0, p.slot_floats, p.M, n_ok, t0, t1, y_out + out_col, ldy);
-        else epi_finish<8>(d_addr, both, c_begin, c_end, keep, S, src0, p.slot_floats, p.M, n_ok, t0, t1, y_out + out_col, ldy);
+        if (wide) epi_finish<16>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, p.M, n_ok, t0, t1, y_out + out_col, ldy);
+        else epi_finish<8>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, p.M, n_ok, t0, t1, y_out + out_col, ldy);
         tc_fence_before();
-        mbar_arrive(bar_d_empty + 8 * buf);
+        __syncwarp();                                          // one arrival per warp, where the issuers wait
+        if (lane == 0) {
+          if (kPair) mbar_arrive_cluster(map_to_rank(bar_d_empty + 8 * buf, 0));
+          else mbar_arrive(bar_d_empty + 8 * buf);
+        }
         if (P.signal) {
           epi_bar();                                           // all stores of the CTA are issued ...
           if (lead) {
@@ -464,12 +555,16 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       // store the partial tile [token][column] (a warp writes 128 contiguous bytes per token), give the
       // accumulator back, count this CTA in
       {
-        float *dst = p.partials + (long long)(s.slot0 + s.contrib_idx) * p.slot_floats + n;
+        float *dst = p.partials + ((long long)tile_mul * (s.slot0 + s.contrib_idx) + rank) * p.slot_floats + n;
         if (wide) epi_store_partial<16>(d_addr, both, c_begin, c_end, p.M, dst);
         else epi_store_partial<8>(d_addr, both, c_begin, c_end, p.M, dst);
       }
       tc_fence_before();
-      mbar_arrive(bar_d_empty + 8 * buf);
+      __syncwarp();
+      if (lane == 0) {
+        if (kPair) mbar_arrive_cluster(map_to_rank(bar_d_empty + 8 * buf, 0));
+        else mbar_arrive(bar_d_empty + 8 * buf);
+      }
       epi_bar();
       if (lead) {
         __threadfence();
@@ -497,7 +592,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
               const int r = r0 + u * nc;
 #pragma unroll
               for (int k = 0; k < 4; ++k)
-                w[u][k] = (r < t1 && i + k < S) ? __ldcg(src0 + (long long)(i + k) * p.slot_floats + r * kTileN) : 0.f;
+                w[u][k] = (r < t1 && i + k < S) ? __ldcg(src0 + (long long)(i + k) * slot_step + r * kTileN) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u)
@@ -523,9 +618,14 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) {          // the leader's MMAs write the peer's tensor memory, the peer arrives on the leader's barriers
+    cluster_arrive();
+    cluster_wait();
+  }
   if (warp == 2) {
     __syncwarp();
-    tmem_dealloc<kPlTmemCols>(tmem);
+    if (kPair) tmem_dealloc_pair<kPlTmemCols>(tmem);
+    else tmem_dealloc<kPlTmemCols>(tmem);
   }
   // the last CTA to leave puts every counter back to zero for the next launch
   if (threadIdx.x == 0) {
@@ -574,9 +674,10 @@ bool plan_encode_x(CUtensorMap *map, const __half *x, int M, long long ldx, int 
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int plan_nw(int MT) {
-  const int budget = kPlSmemBytes - 1024 - kPlStages * MT * 256 - 512;
-  const int nw = budget / kWSlotBytes;
+// ring depth and shared memory for MTL token rows per CTA
+int plan_nw(int MTL) {
+  const int budget = kPlSmemBytes - 1024 - kPlStages * MTL * 256 - 512;
+  const int nw = (budget / kWSlotBytes) & ~3;          // four sub-rings of equal depth, one per team
   return nw > 20 ? 20 : nw;
 }
 
@@ -722,25 +823,80 @@ int plan_build_schedule(const std::vector<PlanGeom> &ops, int n_ctas, const int 
   return ROSAQ_OK;
 }
 
-// CTAs of the persistent grid on the context's device: one per SM (a CTA takes all of an SM's tensor
-// memory and most of its shared memory).
+template <typename K>
+static int plan_launch_kernel(K kern, const PlanLaunch &l, const PlParams &q, size_t smem, cudaStream_t s) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(l.n_ctas, 1, 1);
+  cfg.blockDim = dim3(kPlThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeCooperative;        // all CTAs resident: the waits between CTAs cannot starve
+  attr[na].val.cooperative = 1;
+  ++na;
+  if (l.pair) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 2;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  if (cudaLaunchKernelEx(&cfg, kern, q) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ROSAQ_ERR_CUDA;
+  }
+  return ROSAQ_OK;
+}
+
+// Entries of the schedule = CTAs (one per SM), or, for pairs, clusters of two CTAs that the device keeps
+// resident at once (an SM without a free neighbour in its GPC cannot host half a pair).  0 when pairs are
+// not available.
+int plan_units(rosaq_ctx *ctx, bool pair) {
+  if (ctx->pl_ctas <= 0) {
+    if (plan_set_attrs(linear_plan_kernel<4, false>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<3, false>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<4, true>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<3, true>, kPlSmemBytes) != ROSAQ_OK)
+      return 0;
+    int p = ctx->sm_count;
+    if (p > kPlanMaxCtas) p = kPlanMaxCtas;
+    ctx->pl_ctas = p;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * (p / 2), 1, 1);
+    cfg.blockDim = dim3(kPlThreads);
+    cfg.dynamicSmemBytes = kPlSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, linear_plan_kernel<4, true>, &cfg) != cudaSuccess) {
+      (void)cudaGetLastError();
+      clusters = 0;
+    }
+    if (clusters > p / 2) clusters = p / 2;
+    ctx->pl_pairs = clusters;
+  }
+  return pair ? ctx->pl_pairs : ctx->pl_ctas;
+}
+
 int plan_ctas(rosaq_ctx *ctx) {
-  if (ctx->pl_ctas > 0) return ctx->pl_ctas;
-  if (plan_set_attrs(linear_plan_kernel<4>, kPlSmemBytes) != ROSAQ_OK || plan_set_attrs(linear_plan_kernel<3>, kPlSmemBytes) != ROSAQ_OK)
-    return 0;
-  int p = ctx->sm_count;
-  if (p > kPlanMaxCtas) p = kPlanMaxCtas;
-  ctx->pl_ctas = p;
-  return p;
+  const int pairs = plan_units(ctx, true);
+  return ctx->pl_mode != 1 && pairs > 0 ? 2 * pairs : plan_units(ctx, false);
 }
 
 // Looks the schedule of this geometry up in the context's cache, or builds and uploads it.
-static int plan_get_schedule(rosaq_ctx *ctx, const std::vector<PlanGeom> &geom, const PlanSchedule **out) {
-  const int P = plan_ctas(ctx);
+static int plan_get_schedule(rosaq_ctx *ctx, const std::vector<PlanGeom> &geom, int P, const int *cost,
+                             const PlanSchedule **out) {
   if (P <= 0) return ROSAQ_ERR_CUDA;
   for (PlanSchedule *s : ctx->pl_schedules) {
-    if (s->n_ctas != P || s->geom.size() != geom.size() || s->cost[0] != ctx->pl_cost[0] || s->cost[1] != ctx->pl_cost[1] ||
-        s->cost[2] != ctx->pl_cost[2])
+    if (s->n_ctas != P || s->geom.size() != geom.size() || s->cost[0] != cost[0] || s->cost[1] != cost[1] || s->cost[2] != cost[2])
       continue;
     bool same = true;
     for (size_t i = 0; i < geom.size() && same; ++i)
@@ -754,8 +910,8 @@ static int plan_get_schedule(rosaq_ctx *ctx, const std::vector<PlanGeom> &geom, 
   PlanSchedule *s = new (std::nothrow) PlanSchedule();
   if (!s) return ROSAQ_ERR_ALLOC;
   s->geom = geom;
-  for (int i = 0; i < 3; ++i) s->cost[i] = ctx->pl_cost[i];
-  int st = plan_build_schedule(geom, P, ctx->pl_cost, s);
+  for (int i = 0; i < 3; ++i) s->cost[i] = cost[i];
+  int st = plan_build_schedule(geom, P, cost, s);
   if (st == ROSAQ_OK && s->n_counters > kPlMaxCounters) st = ROSAQ_ERR_UNSUPPORTED_SHAPE;
   if (st == ROSAQ_OK) {
     const size_t seg_bytes = std::max<size_t>(s->segs.size(), 1) * sizeof(PlanSeg), beg_bytes = (size_t)(P + 1) * sizeof(int);
@@ -795,6 +951,11 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
   if (n < 1 || n > kPlanMaxOps || M < 1 || M > kPlTokens) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
   std::vector<PlanGeom> geom(n);
   int bits = 0;
+  // pairs of CTAs (two adjacent column tiles per MMA) unless an operand's adjacent tiles multiply different
+  // channels (a block-diagonal operand with an odd number of groups per block) or pairs are switched off
+  bool pair = ctx->pl_mode != 1 && plan_units(ctx, true) > 0;
+  for (int i = 0; i < n && pair; ++i) pair = ops[i].t->block_groups % 2 == 0;
+  const int tile_div = pair ? 2 : 1;
   for (int i = 0; i < n; ++i) {
     const TiledOperand &t = *ops[i].t;
     const int G = groups_per_tile(t);
@@ -810,14 +971,20 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
     const int rep = ops[i].col_map && G <= 2 ? 4 : 1;
     // (and such a copy keeps the epilogue warps of its CTA busy for about as long as sixteen quantized
     // groups keep the MMA threads: counted as that, so that these tiles spread over many CTAs)
-    geom[i] = PlanGeom{t.n_tiles, G, t.g_fp16, ops[i].dep, rep, rep > 1 ? kPlanCostScatterTile : 0};
+    geom[i] = PlanGeom{(t.n_tiles + tile_div - 1) / tile_div, G, t.g_fp16, ops[i].dep, rep,
+                       rep > 1 ? (pair ? kPlanPairCostScatterTile : kPlanCostScatterTile) : 0};
   }
+  const int dflt_single[3] = {kPlanCostFp16, kPlanCostQuant, kPlanCostTile};
+  const int dflt_pair[3] = {kPlanPairCostFp16, kPlanPairCostQuant, kPlanPairCostTile};
+  const int *cost = ctx->pl_cost_set ? ctx->pl_cost : (pair ? dflt_pair : dflt_single);
   const PlanSchedule *s = nullptr;
-  int st = plan_get_schedule(ctx, geom, &s);
+  int st = plan_get_schedule(ctx, geom, plan_units(ctx, pair), cost, &s);
   if (st != ROSAQ_OK) return st;
-  const int MT = ((M + 15) / 16) * 16;
+  if (tile_div * s->n_counters > kPlMaxCounters) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  const int MT = pair ? ((M + 31) / 32) * 32 : ((M + 15) / 16) * 16;
+  const int MTL = MT / tile_div;                       // token rows a CTA keeps in shared memory
   const int slot_floats = MT * kTileN;
-  const size_t need = (size_t)std::max(s->n_slots, 1) * slot_floats * sizeof(float);
+  const size_t need = (size_t)tile_div * std::max(s->n_slots, 1) * slot_floats * sizeof(float);
   if (ctx->pl_partial_bytes < need) {
     // the old buffer may still be in use by work queued on some stream
     if (cudaDeviceSynchronize() != cudaSuccess) {
@@ -839,7 +1006,7 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
     const TiledOperand &t = *ops[i].t;
     const __half *x = ops[i].dep >= 0 ? ops[ops[i].dep].y : ops[i].x;
     const long long ldx = ops[i].dep >= 0 ? ops[ops[i].dep].ldy : ops[i].ldx;
-    if (!plan_encode_x(&q->xmap[i], x, M, ldx, t.d_in, MT)) {
+    if (!plan_encode_x(&q->xmap[i], x, M, ldx, t.d_in, MTL)) {
       delete q;
       return ROSAQ_ERR_CUDA;
     }
@@ -850,10 +1017,11 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
     P.tile_stride = t.tile_stride;
     P.ldy = ops[i].ldy;
     P.d_out = t.d_out;
+    P.n_tiles = t.n_tiles;
     P.g_fp16 = t.g_fp16;
     P.block_groups = t.block_groups;
     P.dep = ops[i].dep;
-    P.dep_target = ops[i].dep >= 0 ? s->done_target[ops[i].dep] : 0u;
+    P.dep_target = ops[i].dep >= 0 ? (unsigned)tile_div * s->done_target[ops[i].dep] : 0u;   // both CTAs of a pair count
     P.signal = 0;
   }
   for (int i = 0; i < n; ++i)
@@ -864,13 +1032,14 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
   q->sync = ctx->pl_sync;
   q->status = ctx->d_status;
   q->wait_limit = ctx->wait_limit;
-  q->n_counters = s->n_counters;
+  q->n_counters = tile_div * s->n_counters;
   q->M = M;
   q->MT = MT;
-  q->NW = plan_nw(MT);
+  q->NW = plan_nw(MTL);
   q->slot_floats = slot_floats;
   out->params = q;
-  out->n_ctas = s->n_ctas;
+  out->n_ctas = tile_div * s->n_ctas;
+  out->pair = pair;
   out->bits = bits == 3 ? 3 : 4;
   out->partial_bytes = need;
   return ROSAQ_OK;
@@ -887,23 +1056,11 @@ int plan_launch(rosaq_ctx *ctx, const PlanLaunch &l, cudaStream_t s) {
   if (ctx->pl_partial_bytes < l.partial_bytes) return ROSAQ_ERR_INVALID_ARG;
   q->partials = ctx->pl_partials;                      // the workspace may have grown since the plan was made
   q->wait_limit = ctx->wait_limit;
-  const size_t smem = plan_smem_bytes(q->MT, q->NW);
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(l.n_ctas, 1, 1);
-  cfg.blockDim = dim3(kPlThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;         // all CTAs resident: the waits between CTAs cannot starve
-  attr[0].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = l.bits == 3 ? cudaLaunchKernelEx(&cfg, linear_plan_kernel<3>, *q) : cudaLaunchKernelEx(&cfg, linear_plan_kernel<4>, *q);
-  if (e != cudaSuccess) {
-    (void)cudaGetLastError();
-    return ROSAQ_ERR_CUDA;
-  }
-  return ROSAQ_OK;
+  const size_t smem = plan_smem_bytes(l.pair ? q->MT / 2 : q->MT, q->NW);
+  if (l.pair) return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, true>, l, *q, smem, s)
+                                 : plan_launch_kernel(linear_plan_kernel<4, true>, l, *q, smem, s);
+  return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, false>, l, *q, smem, s)
+                     : plan_launch_kernel(linear_plan_kernel<4, false>, l, *q, smem, s);
 }
 
 }  // namespace rosaq

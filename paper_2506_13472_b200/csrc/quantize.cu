@@ -401,13 +401,20 @@ int launch_import(const TiledOperand &t, const uint32_t *qw, const __half *scale
 // =====================================================================================
 __global__ void __launch_bounds__(kTileN)
 rotation_tiles_kernel(const __half *__restrict__ q, int dh, TiledOperand t) {
+  // A column tile holds the groups of its (possibly merged) diagonal block: dm channels = block_groups * 128,
+  // or all of d_in.  When two 128 x 128 head blocks are merged into one 256 x 256 block the off-diagonal
+  // quarters are zero.
   const int nt = blockIdx.x, lg = blockIdx.y, nl = threadIdx.x;
   const int col = nt * kTileN + nl;          // column of blockdiag
   const int h = col / dh, c = col % dh;
+  const int dm = t.block_groups > 0 ? t.block_groups * kGroup : t.d_in;
+  const int k_base = (col / dm) * dm + lg * kGroup;             // first input channel of this group
   const __half *R = q + (long long)h * dh * dh;
   uint8_t *tile = t.blob + tile_offset(t, nt, lg);
-  for (int k = 0; k < kGroup; ++k)
-    *reinterpret_cast<__half *>(tile + fp16_tile_byte(k, nl)) = R[(long long)(lg * kGroup + k) * dh + c];
+  for (int k = 0; k < kGroup; ++k) {
+    const int kg = k_base + k;
+    *reinterpret_cast<__half *>(tile + fp16_tile_byte(k, nl)) = kg / dh == h ? R[(long long)(kg % dh) * dh + c] : __float2half(0.f);
+  }
 }
 
 int launch_rotation_tiles(const __half *q, int d, int n_blocks, const TiledOperand &t, cudaStream_t s) {

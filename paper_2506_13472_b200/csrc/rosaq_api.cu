@@ -133,6 +133,9 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->sk_arrive = nullptr;
   ctx->sk_ctas = 2 * ctx->sm_count < rosaq::kSkMaxCtas ? 2 * ctx->sm_count : rosaq::kSkMaxCtas;
   ctx->pl_ctas = 0;
+  ctx->pl_pairs = 0;
+  ctx->pl_mode = 1;   // pairs of CTAs are built and tested but measured slower so far: off unless asked for
+  ctx->pl_cost_set = 0;
   ctx->pl_cost[0] = kPlanCostFp16, ctx->pl_cost[1] = kPlanCostQuant, ctx->pl_cost[2] = kPlanCostTile;
   ctx->pl_partials = nullptr;
   ctx->pl_partial_bytes = 0;
@@ -387,7 +390,10 @@ int rosaq_rotation_create(rosaq_ctx *ctx, const rosaq_rot *rot, rosaq_rotation *
   r->d = rot->d;
   r->device = ctx->device;
   r->col_map = nullptr;
-  const int bg = dh / kGroup;
+  // 128-channel head blocks are stored in pairs, as 256 x 256 blocks with zero off-diagonal quarters (2 MB
+  // instead of 1 MB at d = 4096): two adjacent column tiles then multiply the same channels, which lets a
+  // pair of SMs share one MMA stream over them
+  const int bg = (dh == kGroup && rot->n_blocks % 2 == 0) ? 2 : dh / kGroup;
   r->t = make_geometry(rot->d, rot->d, 4, bg, 0, rot->n_blocks == 1 ? 0 : bg);
   int st = alloc_blob(&r->t);
   if (st == ROSAQ_OK && rot->perm) {
@@ -584,7 +590,15 @@ int rosaq_set_plan_costs(rosaq_ctx *ctx, int fp16_group, int quant_group, int ti
   if (!ctx || fp16_group < 1 || quant_group < 1 || tile < 0 || fp16_group > 1000 || quant_group > 1000 || tile > 1000)
     return ROSAQ_ERR_INVALID_ARG;
   ctx->pl_cost[0] = fp16_group, ctx->pl_cost[1] = quant_group, ctx->pl_cost[2] = tile;
+  ctx->pl_cost_set = 1;
   return ROSAQ_OK;
+}
+
+int rosaq_set_plan_pairs(rosaq_ctx *ctx, int enable) {
+  if (!ctx) return ROSAQ_ERR_INVALID_ARG;
+  const int prev = ctx->pl_mode != 1;
+  ctx->pl_mode = enable ? 0 : 1;
+  return prev;
 }
 
 int rosaq_plan_ctas(rosaq_ctx *ctx) {

@@ -184,6 +184,9 @@ constexpr int kPlSyncWords = kPlSyncArrive + kPlMaxCounters;
 // output is scattered keeps the epilogue warps busy for about as long as seven quantized groups keep
 // the MMA threads.
 constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 7, kPlanCostTile = 1, kPlanCostScatterTile = 48;
+// With pairs of CTAs a quantized group costs each SM half the MMAs: both kinds of group are then bound by
+// their bytes (32 KB against 8.5 KB).
+constexpr int kPlanPairCostFp16 = 15, kPlanPairCostQuant = 4, kPlanPairCostTile = 1, kPlanPairCostScatterTile = 64;
 
 // One piece of work of a CTA: groups [g_begin, g_end) of column tile `tile` of problem `prob`.
 struct PlanSeg {
@@ -229,6 +232,7 @@ struct PlanOp {
 struct PlanLaunch {
   void *params = nullptr;   // kernel parameters (tensor maps, problem table), owned
   int n_ctas = 0, bits = 4;
+  bool pair = false;        // clusters of two CTAs sharing an MMA stream
   size_t partial_bytes = 0;
 };
 }  // namespace rosaq
@@ -245,8 +249,11 @@ struct rosaq_ctx {
   int *sk_arrive;      // stream-K: per-tile arrival counters, zero between launches
   int sk_ctas;         // CTAs the partial-tile workspace was sized for
   // persistent multi-problem launch
-  int pl_ctas;                                   // CTAs of its grid (0 until first asked for)
-  int pl_cost[3];                                // cost of an fp16 group, a quantized group, a tile's epilogue
+  int pl_ctas;                                   // CTAs of its grid, one per SM (0 until first asked for)
+  int pl_pairs;                                  // clusters of two CTAs the device keeps resident at once
+  int pl_mode;                                   // 0: pairs of CTAs where the operands allow, 1: single CTAs only
+  int pl_cost[3];                                // cost of an fp16 group, a quantized group, a tile's epilogue ...
+  int pl_cost_set;                               // ... when set through rosaq_set_plan_costs, else the defaults
   float *pl_partials;                            // partial tiles exchanged between CTAs; grown on demand
   size_t pl_partial_bytes;
   unsigned *pl_sync;                             // counters, zero between launches
@@ -315,6 +322,7 @@ int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long lo
 
 int plan_build_schedule(const std::vector<PlanGeom> &ops, int n_ctas, const int *cost, PlanSchedule *out);
 int plan_ctas(rosaq_ctx *ctx);
+int plan_units(rosaq_ctx *ctx, bool pair);
 int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *out);
 int plan_launch(rosaq_ctx *ctx, const PlanLaunch &l, cudaStream_t s);
 void plan_release(PlanLaunch *l);

@@ -37,11 +37,13 @@ def householder_rotation(d, seed, key):
     return synth.apply_householders(np.eye(d), vs)
 
 
+@pytest.mark.parametrize("pairs", [True, False])
 @pytest.mark.parametrize("bits,M", [(4, 4), (3, 64), (4, 33), (3, 1)])
-def test_small_layer_plan_against_oracle_and_separate_calls(ctx, bits, M):
+def test_small_layer_plan_against_oracle_and_separate_calls(ctx, bits, M, pairs):
     """A decoder layer in miniature (d = 512, ffn = 1024, 4 heads): dense rotations for the attention and
     MLP inputs, a head-wise one with its permutation for the o_proj input, down_proj un-rotated."""
     d, f = 512, 1024
+    ctx.set_plan_pairs(pairs)
     c, hw = H.config_tiny(), H.config_headwise()
     R2 = householder_rotation(d, 7, "plan-mlp")
     rots = {"attn": ctx.rotation_create(dev(c["R16"])),
@@ -102,6 +104,7 @@ def test_small_layer_plan_against_oracle_and_separate_calls(ctx, bits, M):
     for k in ys:
         assert torch.equal(ys[k].view(torch.int16), first[k].view(torch.int16)), k
     plan.free()
+    ctx.set_plan_pairs(True)
 
 
 def test_plan_argument_errors(ctx):
@@ -123,13 +126,15 @@ def test_plan_argument_errors(ctx):
     assert ctx.last_status() == rb.ROSAQ_OK
 
 
+@pytest.mark.parametrize("pairs", [True, False])
 @pytest.mark.parametrize("bits", [4, 3])
-def test_7b_layer_plan_all_columns(ctx, bits):
+def test_7b_layer_plan_all_columns(ctx, bits, pairs):
     """The benchmark's step: the ten operations of a LLaMA-7B-shaped decoder layer at 64 tokens as one
     launch.  Weights are imported random codes (the quantizer is covered elsewhere); every output column
     is compared with the oracle's forward on the same arrays, fed the rotated activations the GPU
     produced, which are themselves compared with the oracle's x . R."""
     d, f, M = 4096, 11008, 64
+    ctx.set_plan_pairs(pairs)
     g = torch.Generator(device="cuda").manual_seed(17 + bits)
 
     def packed(d_in, d_out):
@@ -183,3 +188,4 @@ def test_7b_layer_plan_all_columns(ctx, bits):
     for k, v in list(ys.items()) + [("xr_" + k, v) for k, v in xr.items()]:
         assert torch.equal(v.view(torch.int16), first[k].view(torch.int16)), k
     plan.free()
+    ctx.set_plan_pairs(True)
