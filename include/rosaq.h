@@ -268,13 +268,13 @@ int rosaq_plan_free(rosaq_plan *plan);
 
 /* Test and tuning hook: the relative cost of an fp16 group, a quantized group and a started tile that
  * rosaq_plan_create (and the single calls, which plan internally) use from now on to cut a phase into
- * equal shares (defaults 10, 7, 1 for single CTAs and 15, 4, 1 for pairs; 1 <= cost <= 1000, tile >= 0).  Changes how K is divided among the CTAs,
- * hence the fp32 summation order of later plans; plans already created keep theirs. */
+ * equal shares (defaults 10, 7, 1 for single CTAs and 15, 4, 1 for pairs; 1 <= cost <= 1000, tile >= 0).
+ * Changes how K is divided among the CTAs, hence the fp32 summation order of later plans; plans already created keep theirs. */
 int rosaq_set_plan_costs(rosaq_ctx *ctx, int fp16_group, int quant_group, int tile);
 
 /* Test and tuning hook: enable != 0 lets the persistent launch run as pairs of CTAs that share one
- * MMA stream over two adjacent column tiles (tcgen05 cta_group::2) wherever the operands allow it; 0 forces
- * single CTAs.  The two cut K differently: results agree to fp32 summation order.  Applies to plans created
+ * MMA stream over two adjacent column tiles (tcgen05 cta_group::2) wherever the operands allow it; 0 (the default)
+ * forces single CTAs.  The two cut K differently: results agree to fp32 summation order.  Applies to plans created
  * afterwards.  Returns the previous setting (1 or 0), or a negative status. */
 int rosaq_set_plan_pairs(rosaq_ctx *ctx, int enable);
 

@@ -104,7 +104,7 @@ def test_small_layer_plan_against_oracle_and_separate_calls(ctx, bits, M, pairs)
     for k in ys:
         assert torch.equal(ys[k].view(torch.int16), first[k].view(torch.int16)), k
     plan.free()
-    ctx.set_plan_pairs(True)
+    ctx.set_plan_pairs(False)
 
 
 def test_plan_argument_errors(ctx):
@@ -188,4 +188,4 @@ def test_7b_layer_plan_all_columns(ctx, bits, pairs):
     for k, v in list(ys.items()) + [("xr_" + k, v) for k, v in xr.items()]:
         assert torch.equal(v.view(torch.int16), first[k].view(torch.int16)), k
     plan.free()
-    ctx.set_plan_pairs(True)
+    ctx.set_plan_pairs(False)
