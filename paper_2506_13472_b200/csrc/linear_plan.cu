@@ -28,19 +28,19 @@
 // returns.  The last CTA to leave clears the counters, so the next launch starts from zero whatever
 // happened.
 //
-// One CTA owns an SM.  At 64 tokens a 128 x 64 x 16 MMA with its weight operand in tensor memory occupies
-// the tensor pipe for about 45 cycles, eight of them per 128-channel group: 360 cycles, as long as the
-// group's bytes take to arrive from HBM.  Two CTAs per SM only take turns on that pipe and lengthen each
-// other's dequantise -> MMA -> release chain (measured: 1330 cycles per group and CTA with two operand
-// buffers each).  In place, however, one thread needs 600 to 700 cycles to issue the eight MMAs and the
-// commit of a group (also when nothing else runs on the SM), while two threads issuing to different
-// accumulators overlap.  So one CTA with TWO MMA-issuing threads: groups with an even position in the
-// CTA's stream accumulate into one tile, odd ones into another, and the epilogue adds the two.
-// Warp 0 = weight-tile producer (bulk copies, L2 evict-first), 1 = activation producer (TMA), 2 and 3 =
-// MMA issuers (2 also owns the tensor memory), 4..19 = four dequantisation teams (group j goes to team and
-// operand buffer j mod 4), 20..27 = epilogue (two warps per TMEM lane quadrant, half of the tokens each).
-// Tensor memory (512 columns): accumulators of piece parity b and issuer i at (2b + i) * 64, operand
-// buffers from 256.
+// One CTA owns an SM.  A tcgen05.mma of 128 x N x 16 costs 55 cycles of the tensor pipe for every N <= 64
+// (measured back to back), eight of them per 128-channel group: 440 cycles, 542 with the group's commit,
+// against 375 cycles for the group's bytes from HBM.  Two CTAs per SM only take turns on that pipe and
+// lengthen each other's dequantise -> MMA -> release chain; one CTA with one issuing thread spent 900
+// cycles per group in place, with TWO issuing threads 700: groups with an even position in the CTA's stream
+// accumulate into one tile, odd ones into another, and the epilogue adds the two.  Instruction issue
+// comes next (1700 warp instructions per group = 430 cycles of the four schedulers), which is why every
+// role walks only over its own groups and the epilogue loops carry no per-element address arithmetic.
+// Warp 0 = weight-tile producer (bulk copies, L2 evict-first; one sub-ring of slots per team), 1 =
+// activation producer (TMA), 2 and 3 = MMA issuers (2 also owns the tensor memory), 4..19 = four
+// dequantisation teams (group j goes to team and operand buffer j mod 4), 20..27 = epilogue (two warps per
+// TMEM lane quadrant, half of the tokens each).  Tensor memory (512 columns): accumulators of piece parity b
+// and issuer i at (2b + i) * 64, operand buffers from 256.
 #include <cuda.h>
 
 #include <algorithm>
@@ -55,7 +55,9 @@ namespace {
 
 constexpr int kPlTmemCols = 512;
 constexpr int kPlTeams = 4;                         // dequantisation teams of four warps
-constexpr int kPlStages = kPlTeams;                 // TMEM operand buffers, each with its activation slot: one per team
+constexpr int kPlStages = kPlTeams;                 // TMEM operand buffers, each with its activation slot: one per team ...
+constexpr int kPlPairStages = 6;                    // ... six in a pair of CTAs (one issuing thread, two accumulators)
+constexpr int kPlMaxStages = 6;
 constexpr int kPlTokens = 64;                       // token capacity of an accumulator and of a partial tile
 constexpr int kPlFirstDequantWarp = 4, kPlFirstEpiWarp = kPlFirstDequantWarp + 4 * kPlTeams;
 constexpr int kPlEpiThreads = 256;                  // two warps per TMEM lane quadrant
@@ -222,12 +224,17 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
   const int MTL = kPair ? MT >> 1 : MT;                        // token rows this CTA keeps in shared memory
   const uint32_t x_slot_bytes = (uint32_t)MTL * 256u;
   const uint32_t x_ring = base;
-  const uint32_t w_ring = x_ring + kPlStages * x_slot_bytes;
+  // operand buffers: a single CTA has two issuing threads with an accumulator each per piece parity (256
+  // columns) and one buffer per team; a pair has one issuing thread (an MMA over both SMs costs no more than
+  // one over one) and spends the columns on two more buffers, which hides the longer chain of a pair
+  // (dequantise -> remote arrive -> MMA -> multicast commit)
+  constexpr int NS = kPair ? kPlPairStages : kPlStages;
+  const uint32_t w_ring = x_ring + NS * x_slot_bytes;
   const uint32_t bars = w_ring + p.NW * kWSlotBytes;
   const uint32_t bar_w_full = bars, bar_w_empty = bar_w_full + 8 * p.NW;
   const uint32_t bar_a_full = bar_w_empty + 8 * p.NW;          // operand buffer written + activation slot landed
-  const uint32_t bar_s_empty = bar_a_full + 8 * kPlStages;     // stage consumed by its MMAs
-  const uint32_t bar_d_full = bar_s_empty + 8 * kPlStages;     // accumulator complete (two accumulators)
+  const uint32_t bar_s_empty = bar_a_full + 8 * kPlMaxStages;  // stage consumed by its MMAs
+  const uint32_t bar_d_full = bar_s_empty + 8 * kPlMaxStages;  // accumulator complete (two accumulators)
   const uint32_t bar_d_empty = bar_d_full + 16;                // accumulator drained
   const uint32_t bar_drain = bar_d_empty + 16;                 // two: one per issuer
   const uint32_t misc = bar_drain + 16;                         // [0] TMEM base, [1] abort flag, [2] last CTA out
@@ -247,13 +254,13 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       mbar_init(bar_w_full + 8 * i, 1);
       mbar_init(bar_w_empty + 8 * i, kTeamThreads);
     }
-    for (int i = 0; i < kPlStages; ++i) {
+    for (int i = 0; i < NS; ++i) {
       // a team's arrivals (per thread; in a pair per warp, from both CTAs) + the activation copy
       mbar_init(bar_a_full + 8 * i, (kPair ? 2 * (kTeamThreads / 32) : kTeamThreads) + 1);
       mbar_init(bar_s_empty + 8 * i, 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_d_full + 8 * i, 2);                        // both issuers
+      mbar_init(bar_d_full + 8 * i, kPair ? 1 : 2);            // the issuing threads
       mbar_init(bar_d_empty + 8 * i, (kPair ? 2 : 1) * (kPlEpiThreads / 32));   // one arrival per epilogue warp
       mbar_init(bar_drain + 8 * i, 1);
     }
@@ -274,7 +281,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
   }
   tc_fence_after();
   const uint32_t tmem = misc_ptr[0];
-  const uint32_t a_col0 = 4 * kPlTokens;
+  const uint32_t a_col0 = (kPair ? 2 : 4) * kPlTokens;         // operand buffers follow the accumulators
   const int qbytes = quant_tile_bytes(kBits);
 
   if (warp == 0) {
@@ -357,7 +364,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         // block-diagonal operand: a column tile only multiplies the channels of its own diagonal block
         const int g_block0 = P.block_groups > 0 ? ((tile_mul * s.tile + (int)rank) / P.block_groups) * P.block_groups : 0;
         const CUtensorMap *map = &p.xmap[s.prob];
-        for (int g = s.g_begin; g < s.g_end; ++g, ++gc, rs.advance(kPlStages)) {
+        for (int g = s.g_begin; g < s.g_end; ++g, ++gc, rs.advance(NS)) {
           const int slot = rs.idx;
           if (!ab.wait(bar_s_empty + 8 * slot, rs.lap ^ 1u)) {
             live = false;
@@ -377,10 +384,10 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       // (in a pair the leader's barriers count the copies of both CTAs, and the peer stays until the cluster
       // barrier at the end of the kernel, which the leader reaches after this drain)
       if (ab.set() && is_lead) {
-        for (int back = 1; back <= kPlStages && back <= gc; ++back) {
+        for (int back = 1; back <= NS && back <= gc; ++back) {
           const int u = gc - back;
           for (int it = 0; it < kDrainPolls; ++it)
-            if (ab.poll(bar_a_full + 8 * (u % kPlStages), (u / kPlStages) & 1)) break;
+            if (ab.poll(bar_a_full + 8 * (u % NS), (u / NS) & 1)) break;
         }
       }
     }
@@ -389,8 +396,9 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
     // j mod 2 == i (operand buffers i and i + 2) and accumulates them into its own tile; per group one
     // wait, eight MMAs, one commit.  Every piece is committed by both (an issuer without a group in a
     // one-group piece arrives by hand), so the epilogue waits for one barrier.
-    if (lane == 0 && is_lead) {
+    if (lane == 0 && is_lead && !(kPair && warp == 3)) {       // (a pair has one issuing thread)
       const int me = warp - 2;
+      constexpr int kStep = kPair ? 1 : 2;                     // issuers that share the stream
       // M = 128 output columns (256 for a pair), N = MT tokens
       const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | ((kPair ? 16u : 8u) << 24);
       const uint64_t desc0 = make_b_desc(x_ring);
@@ -402,14 +410,14 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         const int buf = nseg & 1;
         if (!ab.wait(bar_d_empty + 8 * buf, ((nseg >> 1) & 1) ^ 1u)) break;   // the piece before last has been drained
         tc_fence_after();
-        const uint32_t d_tmem = tmem + (uint32_t)(2 * buf + me) * kPlTokens;
+        const uint32_t d_tmem = tmem + (uint32_t)(kPair ? buf : 2 * buf + me) * kPlTokens;
         uint32_t accumulate = 0;
-        const int g_first = s.g_begin + ((me - j) & 1), j_base = j - s.g_begin;
+        const int g_first = kPair ? s.g_begin : s.g_begin + ((me - j) & 1), j_base = j - s.g_begin;
         j += s.g_end - s.g_begin;
-        for (int g = g_first; g < s.g_end; g += 2) {
+        for (int g = g_first; g < s.g_end; g += kStep) {
           const int j = j_base + g;
-          const int st = j & (kPlStages - 1);
-          if (!ab.wait(bar_a_full + 8 * st, (uint32_t)(j >> 2) & 1u)) {
+          const int st = j % NS;                               // (a constant: a mask or a multiply)
+          if (!ab.wait(bar_a_full + 8 * st, (uint32_t)(j / NS) & 1u)) {
             live = false;
             break;
           }
@@ -454,8 +462,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
     const int NWT = p.NW >> 2;
     const uint32_t my_ring = w_ring + team * NWT * kWSlotBytes, my_full = bar_w_full + 8 * team * NWT,
                    my_empty = bar_w_empty + 8 * team * NWT;
-    const uint32_t a_addr = lane_addr + a_col0 + team * 64;
-    const uint32_t my_s_empty = bar_s_empty + 8 * team, my_a_full = bar_a_full + 8 * team;
+
     Ring rw{0, 0};
     bool ok = true;
     int j0 = 0;                                      // position of the piece's first group in the CTA's stream
@@ -465,7 +472,10 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       for (int g = s.g_begin + ((team - j0) & (kPlTeams - 1)); g < s.g_end && ok; g += kPlTeams) {
         const bool f16 = g < g_fp16;
         const int nsub = f16 ? 4 : 1;
-        const uint32_t use = (uint32_t)(j0 + g - s.g_begin) >> 2;        // how often this team's buffer was used before
+        const uint32_t j = (uint32_t)(j0 + g - s.g_begin);
+        const uint32_t st = j % NS, use = j / NS;                          // the group's buffer; how often it was used before
+        const uint32_t a_addr = lane_addr + a_col0 + st * 64;
+        const uint32_t my_s_empty = bar_s_empty + 8 * st, my_a_full = bar_a_full + 8 * st;
         bool got = ab.wait(my_s_empty, (use & 1u) ^ 1u);
         for (int sub = 0; sub < nsub && ok; ++sub, rw.advance(NWT)) {
           got = got && ab.wait_local(my_full + 8 * rw.idx, rw.lap);
@@ -506,14 +516,14 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       const PlProblem &P = p.prob[s.prob];
       const int buf = nseg & 1;
       // the piece's groups have positions j0 .. in the CTA's stream: even ones went to issuer 0's tile
-      const bool both = s.g_end - s.g_begin > 1;
-      const int first_acc = both ? 0 : (j0 & 1);
+      const bool both = !kPair && s.g_end - s.g_begin > 1;
+      const int first_acc = (both || kPair) ? 0 : (j0 & 1);
       j0 += s.g_end - s.g_begin;
       bool have_d = ab.wait(bar_d_full + 8 * buf, (nseg >> 1) & 1);
       have_d = __all_sync(0xffffffffu, have_d && !ab.set());
       if (!have_d) break;
       tc_fence_after();
-      const uint32_t d_addr = lane_addr + (uint32_t)(2 * buf + first_acc) * kPlTokens;
+      const uint32_t d_addr = lane_addr + (uint32_t)(kPair ? buf : 2 * buf + first_acc) * kPlTokens;
       const int n_glob = (tile_mul * s.tile + (int)rank) * kTileN + n;
       const bool n_ok = n_glob < P.d_out;
       const long long out_col = n_ok ? (P.col_map ? P.col_map[n_glob] : n_glob) : 0;
@@ -675,14 +685,14 @@ bool plan_encode_x(CUtensorMap *map, const __half *x, int M, long long ldx, int 
 }
 
 // ring depth and shared memory for MTL token rows per CTA
-int plan_nw(int MTL) {
-  const int budget = kPlSmemBytes - 1024 - kPlStages * MTL * 256 - 512;
+int plan_nw(int MTL, int ns) {
+  const int budget = kPlSmemBytes - 1024 - ns * MTL * 256 - 512;
   const int nw = (budget / kWSlotBytes) & ~3;          // four sub-rings of equal depth, one per team
   return nw > 20 ? 20 : nw;
 }
 
-size_t plan_smem_bytes(int MT, int NW) {
-  return 1024 + (size_t)kPlStages * MT * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NW + 2 * kPlStages + 6) + 16;
+size_t plan_smem_bytes(int MTL, int NW, int ns) {
+  return 1024 + (size_t)ns * MTL * 256 + (size_t)NW * kWSlotBytes + 8 * (2 * NW + 2 * kPlMaxStages + 6) + 16;
 }
 
 template <typename K>
@@ -1035,7 +1045,7 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
   q->n_counters = tile_div * s->n_counters;
   q->M = M;
   q->MT = MT;
-  q->NW = plan_nw(MTL);
+  q->NW = plan_nw(MTL, pair ? kPlPairStages : kPlStages);
   q->slot_floats = slot_floats;
   out->params = q;
   out->n_ctas = tile_div * s->n_ctas;
@@ -1056,7 +1066,7 @@ int plan_launch(rosaq_ctx *ctx, const PlanLaunch &l, cudaStream_t s) {
   if (ctx->pl_partial_bytes < l.partial_bytes) return ROSAQ_ERR_INVALID_ARG;
   q->partials = ctx->pl_partials;                      // the workspace may have grown since the plan was made
   q->wait_limit = ctx->wait_limit;
-  const size_t smem = plan_smem_bytes(l.pair ? q->MT / 2 : q->MT, q->NW);
+  const size_t smem = plan_smem_bytes(l.pair ? q->MT / 2 : q->MT, q->NW, l.pair ? kPlPairStages : kPlStages);
   if (l.pair) return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, true>, l, *q, smem, s)
                                  : plan_launch_kernel(linear_plan_kernel<4, true>, l, *q, smem, s);
   return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, false>, l, *q, smem, s)

@@ -184,9 +184,9 @@ constexpr int kPlSyncWords = kPlSyncArrive + kPlMaxCounters;
 // output is scattered keeps the epilogue warps busy for about as long as seven quantized groups keep
 // the MMA threads.
 constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 7, kPlanCostTile = 1, kPlanCostScatterTile = 48;
-// With pairs of CTAs a quantized group costs each SM half the MMAs: both kinds of group are then bound by
-// their bytes (32 KB against 8.5 KB).
-constexpr int kPlanPairCostFp16 = 15, kPlanPairCostQuant = 4, kPlanPairCostTile = 1, kPlanPairCostScatterTile = 64;
+// Pairs of CTAs: a quantized group costs each SM half the MMAs, but the measured layer step is again
+// shortest near 10 : 7 (76 us; 85 us at 12 : 4, 90 us at 15 : 4) -- a pair is not bound by its bytes either.
+constexpr int kPlanPairCostFp16 = 10, kPlanPairCostQuant = 7, kPlanPairCostTile = 1, kPlanPairCostScatterTile = 64;
 
 // One piece of work of a CTA: groups [g_begin, g_end) of column tile `tile` of problem `prob`.
 struct PlanSeg {
