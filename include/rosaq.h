@@ -241,8 +241,10 @@ int rosaq_linear_multi(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const 
  *   op.x_from    -1, or the index (smaller than this operation's) of the operation whose y is this one's
  *                input (a rotation feeding its linears); that y must have this operation's d_in columns
  *   op.y, ldy    DEVICE [M][ldy] fp16 output; the first d_out columns of each row are written
- * Operations without x_from are independent of each other and may run in any order or at the same time;
- * the caller guarantees that no y overlaps any other operation's x or y.  All quantized weights of a list
+ * Operations without x_from are independent of each other and may run in any order or at the same time:
+ * a y that overlaps another operation's y, or any x other than through x_from (its own operation's x
+ * included), is rejected with ROSAQ_ERR_INVALID_ARG (column ranges of one wider buffer with the same row
+ * stride do not overlap; views with different row strides must not share any address range).  All quantized weights of a list
  * have the same bit width.  1 <= M <= 64 and 1 <= n_ops <= 12, otherwise ROSAQ_ERR_UNSUPPORTED_SHAPE.
  * Each y is the sum rosaq_linear computes, added in an order that depends on how the list is divided
  * among the CTAs: results agree with the separate calls to fp32 summation order (a few 1e-5 relative) and

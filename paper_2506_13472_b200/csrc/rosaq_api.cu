@@ -560,6 +560,28 @@ int rosaq_plan_create(rosaq_ctx *ctx, int M, int n_ops, const rosaq_op *ops, ros
       pl->ops.push_back(PlanOp{static_cast<const __half *>(x), ldx, o.x_from >= 0 ? o.x_from : -1, &t,
                                o.r ? o.r->col_map : nullptr, static_cast<__half *>(o.y), o.ldy});
   }
+  // an output may be read only through x_from (which orders the two operations) and written by one
+  // operation: any other overlap of a y with an x or a y would be a race inside the launch
+  // (views of M rows: with equal row strides, disjoint column ranges of one wider buffer do not overlap)
+  auto overlap = [M](const void *pa, int64_t lda, int da, const void *pb, int64_t ldb, int db) {
+    const char *alo = static_cast<const char *>(pa), *blo = static_cast<const char *>(pb);
+    const char *ahi = alo + sizeof(__half) * ((size_t)(M - 1) * (size_t)lda + (size_t)da);
+    const char *bhi = blo + sizeof(__half) * ((size_t)(M - 1) * (size_t)ldb + (size_t)db);
+    if (!(alo < bhi && blo < ahi)) return false;
+    if (lda != ldb) return true;
+    const long long off = (blo - alo) / (long long)sizeof(__half);
+    const long long c = ((off % lda) + lda) % lda;              // b's first column inside a's rows
+    return !(c >= da && c + db <= lda);
+  };
+  for (int i = 0; i < n_ops && st == ROSAQ_OK; ++i) {
+    const PlanOp &a = pl->ops[i];
+    for (int j = 0; j < n_ops && st == ROSAQ_OK; ++j) {
+      const PlanOp &b = pl->ops[j];
+      // (an operation's own x too: its tiles read all of x while others already write y)
+      if (b.dep != i && overlap(a.y, a.ldy, a.t->d_out, b.x, b.ldx, b.t->d_in)) st = ROSAQ_ERR_INVALID_ARG;
+      if (j > i && overlap(a.y, a.ldy, a.t->d_out, b.y, b.ldy, b.t->d_out)) st = ROSAQ_ERR_INVALID_ARG;
+    }
+  }
   if (st == ROSAQ_OK) {
     DeviceGuard guard(ctx->device);
     st = guard.ok ? plan_prepare(ctx, M, n_ops, pl->ops.data(), &pl->launch) : ROSAQ_ERR_CUDA;

@@ -119,6 +119,19 @@ def test_plan_argument_errors(ctx):
         with pytest.raises(rb.RosaqError) as e:
             ctx.plan_create(M, ops)
         assert e.value.status == status
+    # races inside one launch: two operations writing one y, a y that is another operation's plain x,
+    # an operation writing over its own input
+    xs = torch.zeros((8, 256), dtype=torch.float16, device="cuda")
+    wide = torch.zeros((8, 256), dtype=torch.float16, device="cuda")
+    w_sq = ctx.quantize(torch.zeros((128, 128), dtype=torch.float16, device="cuda"), None, bits=4, k_salient=128)
+    for ops in ([(x, None, w4, y), (xs, None, w4, y)],
+                [(x, None, w4, wide[:, :128]), (wide[:, 64:192], None, w_sq, y2)],
+                [(wide[:, :128], None, w_sq, wide[:, 64:192])]):
+        with pytest.raises(rb.RosaqError) as e:
+            ctx.plan_create(8, ops)
+        assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
+    # column ranges of one wider buffer are distinct outputs
+    ctx.plan_create(8, [(x, None, w4, wide[:, :128]), (xs, None, w4, wide[:, 128:])]).free()
     x65 = torch.zeros((65, 256), dtype=torch.float16, device="cuda")
     with pytest.raises(rb.RosaqError) as e:
         ctx.plan_create(65, [(x65, None, w4, empty(65, 128))])
