@@ -677,6 +677,10 @@ def extras(line, args, ctx, rb, model, layers, runners, x, peaks, ms_per_step):
                     "gemm_stage_int4": gemm_stage_table(ctx, m13, 4, peaks, Ms=(1, 64, 512), reps=8),
                     "gemm_stage_int3": gemm_stage_table(ctx, m13, 3, peaks, Ms=(1, 64, 512), reps=8, with_cublas=False),
                     "calib_cov": calib_stream(ctx, peaks)})
+    # prefill-sized batches: from a few hundred tokens on rosaq_linear runs 256 x 256 tiles on pairs of CTAs
+    configs.append({"config": "prefill: 13B and 7B shapes, INT4, M in {1024, 2048}",
+                    "gemm_stage_13b": gemm_stage_table(ctx, m13, 4, peaks, Ms=(1024, 2048), reps=5),
+                    "gemm_stage_7b": gemm_stage_table(ctx, model, 4, peaks, Ms=(1024, 2048), reps=5)})
     line["configs"] = configs
 
 

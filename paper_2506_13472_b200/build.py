@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librosaq.so")
-SOURCES = ["rosaq_api.cu", "quantize.cu", "calib_cov.cu", "linear_simt.cu", "linear_tc.cu", "linear_plan.cu", "linear_static.cu"]
+SOURCES = ["rosaq_api.cu", "quantize.cu", "calib_cov.cu", "linear_simt.cu", "linear_tc.cu", "linear_plan.cu", "linear_prefill.cu", "linear_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -62,9 +62,21 @@ int ensure_workspace(rosaq_ctx *ctx, size_t bytes, cudaStream_t s) {
   return ROSAQ_OK;
 }
 
+constexpr int kPrefillMinTiles = 40, kPrefillMinUnits = 36;
+
 int run_gemm(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t, const int32_t *col_map,
              __half *y, long long ldy, cudaStream_t s) {
   if (ctx->impl == 1) return launch_linear_simt(ctx, x, M, ldx, t, col_map, y, ldy, s);
+  // Large batches of tokens run a weight on 256-column x 256-token tiles shared by pairs of CTAs -- where
+  // the launch is long enough to pay for the exchange of the tiles that two pairs share: at least
+  // kPrefillMinTiles tiles and kPrefillMinUnits 128-channel groups per pair of SMs (measured against the
+  // per-call kernel on the 7B and 13B shapes at 256 ... 2048 tokens).
+  if (prefill_supported(t, col_map) && (ctx->impl == 5 || (ctx->impl == 0 && M > 256))) {
+    const long long tiles = (long long)((t.n_tiles + 1) / 2) * ((M + 255) / 256);
+    const long long units = tiles * groups_per_tile(t);
+    if (ctx->impl == 5 || (tiles >= kPrefillMinTiles && units >= (long long)kPrefillMinUnits * (ctx->sm_count / 2)))
+      return launch_linear_prefill(ctx, x, M, ldx, t, y, ldy, s);
+  }
   return launch_linear_tc(ctx, x, M, ldx, t, col_map, y, ldy, s);
 }
 
@@ -140,6 +152,9 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->pl_partials = nullptr;
   ctx->pl_partial_bytes = 0;
   ctx->pl_sync = nullptr;
+  ctx->pf_pairs = 0;
+  ctx->pf_flags = nullptr;
+  ctx->pf_epoch = 0;
   st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 2 * sizeof(int)));   // [1]: scratch flag of argument checks
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, 2 * sizeof(int)));
   // the stream-K workspace is taken here, once, so that no linear call ever allocates for it
@@ -149,6 +164,8 @@ int rosaq_create(rosaq_ctx **out, int device) {
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->pl_sync), rosaq::kPlSyncWords * sizeof(unsigned)));
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->pl_sync, 0, rosaq::kPlSyncWords * sizeof(unsigned)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->pf_flags), (size_t)ctx->sm_count * sizeof(unsigned)));
+  if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->pf_flags, 0, (size_t)ctx->sm_count * sizeof(unsigned)));
   // the partial tiles of a launch whose CTAs all share tiles at both ends of two phases (grown if a plan needs more)
   if (st == ROSAQ_OK) {
     const size_t bytes = (size_t)4 * ctx->sk_ctas * rosaq::kSkPartialBytes;
@@ -157,6 +174,7 @@ int rosaq_create(rosaq_ctx **out, int device) {
   }
   if (st != ROSAQ_OK) {
     if (ctx->pl_sync) (void)cudaFree(ctx->pl_sync);
+    if (ctx->pf_flags) (void)cudaFree(ctx->pf_flags);
     if (ctx->pl_partials) (void)cudaFree(ctx->pl_partials);
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
     if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
@@ -178,6 +196,7 @@ int rosaq_destroy(rosaq_ctx *ctx) {
     if (ctx->sk_partials) (void)cudaFree(ctx->sk_partials);
     if (ctx->sk_arrive) (void)cudaFree(ctx->sk_arrive);
     if (ctx->pl_sync) (void)cudaFree(ctx->pl_sync);
+    if (ctx->pf_flags) (void)cudaFree(ctx->pf_flags);
     if (ctx->pl_partials) (void)cudaFree(ctx->pl_partials);
     plan_free_schedules(ctx);
     (void)cudaGetLastError();
@@ -218,7 +237,7 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
   if (!ctx) return 0;
   int prev = ctx->impl;
-  if (impl >= 0 && impl <= 4) ctx->impl = impl;
+  if (impl >= 0 && impl <= 5) ctx->impl = impl;
   return prev;
 }
 

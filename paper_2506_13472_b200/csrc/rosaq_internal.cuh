@@ -244,7 +244,8 @@ struct rosaq_ctx {
   void *ws;            // rotated-activation workspace
   size_t ws_bytes;
   long long wait_limit;
-  int impl;            // 0 tensor-core, 1 CUDA-core, 2 tensor-core with CTA pairs, 3 tensor-core without stream-K
+  int impl;            // 0 tensor-core, 1 CUDA-core, 2 tensor-core with CTA pairs, 3 tensor-core without stream-K,
+                       // 4 persistent launch for every call, 5 prefill tiles for every weight
   float *sk_partials;  // stream-K: fp32 partial tiles, [sk_ctas][2][64 tokens][128 columns]
   int *sk_arrive;      // stream-K: per-tile arrival counters, zero between launches
   int sk_ctas;         // CTAs the partial-tile workspace was sized for
@@ -258,6 +259,10 @@ struct rosaq_ctx {
   size_t pl_partial_bytes;
   unsigned *pl_sync;                             // counters, zero between launches
   std::vector<rosaq::PlanSchedule *> pl_schedules;   // one per geometry seen, owned
+  // prefill tiles (pairs of CTAs; the partial tiles of a launch live in pl_partials)
+  int pf_pairs;                                  // pairs the device keeps resident at once (0 until first asked for)
+  unsigned *pf_flags;                            // [pair][rank]: number of the launch whose partial tile is stored
+  unsigned pf_epoch;                             // number of the last launch
 };
 
 struct rosaq_weight {
@@ -319,6 +324,10 @@ int launch_linear_tc(const rosaq_ctx *ctx, const __half *x, int M, long long ldx
 int launch_linear_tc_multi(const rosaq_ctx *ctx, const __half *x, int M, long long ldx, int n,
                            const TiledOperand *const *ts, const int32_t *col_map, __half *const *ys,
                            const long long *ldys, cudaStream_t s);
+
+bool prefill_supported(const TiledOperand &t, const int32_t *col_map);
+int launch_linear_prefill(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t, __half *y,
+                          long long ldy, cudaStream_t s);
 
 int plan_build_schedule(const std::vector<PlanGeom> &ops, int n_ctas, const int *cost, PlanSchedule *out);
 int plan_ctas(rosaq_ctx *ctx);

@@ -138,21 +138,21 @@ def run_linear_case(ctx, x16, W16, Rb32, Rb16, perm, bits, k_salient, impl):
         ctx.set_linear_impl(0)
 
 
-@pytest.mark.parametrize("impl", [1, 0, 4])
+@pytest.mark.parametrize("impl", [1, 0, 4, 5])
 @pytest.mark.parametrize("bits", [4, 3])
 def test_linear_tiny_config(ctx, bits, impl):
     c = H.config_tiny()
     run_linear_case(ctx, c["x"], c["W"], c["R32"], c["R16"], None, bits, 128, impl)
 
 
-@pytest.mark.parametrize("impl", [1, 0, 4])
+@pytest.mark.parametrize("impl", [1, 0, 4, 5])
 @pytest.mark.parametrize("bits", [4, 3])
 def test_linear_headwise(ctx, bits, impl):
     c = H.config_headwise()
     run_linear_case(ctx, c["x"], c["W"], c["Rb32"], c["Rb16"], c["perm"], bits, 128, impl)
 
 
-@pytest.mark.parametrize("impl", [1, 0, 4])
+@pytest.mark.parametrize("impl", [1, 0, 4, 5])
 @pytest.mark.parametrize("M,d_in,d_out,bits,k_salient", [
     (1, 256, 8, 4, 128), (3, 256, 136, 3, 0), (17, 384, 128, 4, 384), (64, 1024, 640, 4, 128),
     (130, 512, 256, 3, 128), (257, 256, 200, 4, 0)])
@@ -160,6 +160,33 @@ def test_linear_shapes_no_rotation(ctx, M, d_in, d_out, bits, k_salient, impl):
     W = synth.weights(d_in, d_out, seed=31, key=f"s{d_in}x{d_out}", outlier_frac=0.01)
     x = synth.rng_for(31, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
     run_linear_case(ctx, x, W, None, None, None, bits, k_salient, impl)
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("M,d_in,d_out,k_salient", [(600, 1024, 1152, 128), (256, 2048, 256, 256), (129, 512, 384, 0)])
+def test_linear_prefill_tiles(ctx, M, d_in, d_out, k_salient, bits):
+    """256-column x 256-token tiles on pairs of CTAs (implementation 5 takes them at every size): several
+    token blocks with a ragged last one, an odd number of 128-column tiles (the second CTA of the last pair
+    has no tile of its own), two salient fp16 groups, none.  Every column against the oracle; the same bits on a
+    second run; agreement with the per-call kernel to fp32 summation order."""
+    W = synth.weights(d_in, d_out, seed=57, key=f"pf{d_in}x{d_out}", outlier_frac=0.01)
+    x = synth.rng_for(57, "x", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+    w = ctx.quantize(dev(W), None, bits=bits, k_salient=k_salient)
+    qd = H.oracle_quantized(W, None, None, bits, k_salient)
+    y0 = ctx.linear(dev(x), w, None).cpu().numpy()
+    ctx.set_linear_impl(5)
+    try:
+        out = torch.full((M + 1, d_out + 8), 7.0, dtype=torch.float16, device="cuda")     # a wider, longer buffer
+        y = ctx.linear(dev(x), w, None, out=out[:M, :d_out]).cpu().numpy()
+        check_status(ctx)
+        again = ctx.linear(dev(x), w, None).cpu().numpy()
+    finally:
+        ctx.set_linear_impl(0)
+    assert np.all(out[M:].cpu().numpy() == 7.0) and np.all(out[:, d_out:].cpu().numpy() == 7.0)   # nothing written outside
+    assert H.rel_fro(y, orc.forward(x, qd, None)) <= H.REL_TOL_Y
+    assert np.array_equal(again.view(np.uint16), y.view(np.uint16))
+    assert H.rel_fro(y, y0.astype(np.float64)) <= 2e-4
+    w.free()
 
 
 def test_linear_strided_activations_and_output(ctx):
@@ -362,7 +389,8 @@ def test_a_perm_that_is_not_a_permutation_is_a_status_code(ctx):
 
 
 # --------------------------------------------------------------------------- bounded waits
-@pytest.mark.parametrize("impl,d_in,d_out", [(3, 1024, 512), (0, 1024, 150 * 128), (4, 1024, 512), (4, 512, 512)])
+@pytest.mark.parametrize("impl,d_in,d_out", [(3, 1024, 512), (0, 1024, 150 * 128), (4, 1024, 512), (4, 512, 512),
+                                               (5, 1024, 512)])
 def test_expired_waits_in_the_linear_kernels_leave_the_context_usable(ctx, impl, d_in, d_out):
     """With the wait limit cut to one poll the linear kernels (cluster split-K, equal shares with the
     workspace exchange, the persistent launch with and without a rotation) may give up anywhere: they must
