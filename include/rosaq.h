@@ -103,7 +103,9 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations);
  * weight stream per SM with the partial tiles exchanged through a workspace that
  * rosaq_create allocated; again the same sums in another order); 4 = every call of up to 64 tokens runs as
  * ONE persistent launch, the rotation and the linears that consume it included (the kernel of rosaq_plan;
- * for a single call slower than 0, which is why it is not the default -- see rosaq_plan_create).
+ * for a single call slower than 0, which is why it is not the default -- see rosaq_plan_create);
+ * 5 = every weight, at any token count, on the 256-column x 256-token tiles that 0 picks for large batches
+ * (rotations and all-fp16 weights stay on the kernels of 0).
  * Returns the previous value. */
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl);
 
@@ -212,6 +214,13 @@ int rosaq_rotate(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_
  *   r != NULL : x . R goes through the context workspace (grown on demand: this call
  *               may then allocate and synchronize once), then the GEMM stage runs
  * Only the first d_out columns of each y row are written.  ldx, ldy multiples of 8.
+ * Any M >= 1.  The kernel is chosen by size: up to 64 tokens the weight-streaming kernels; large batches
+ * (more than 256 tokens, when the launch has at least 40 tiles of 256 columns x 256 tokens and 36
+ * 128-channel groups of work per pair of SMs) run on those tiles, each shared by two CTAs on adjacent SMs
+ * (tcgen05 cta_group::2, one dequantisation of a weight tile per 256 tokens); everything in between one
+ * 128-token tile per CTA.  The choice changes the order of the fp32 sums only; a call gives the same bits
+ * every time.  Calls of one context that use the exchange workspace (the large-batch tiles, the
+ * equal-share kernel, rosaq_plan_run) must not overlap on the GPU: keep them on one stream.
  */
 int rosaq_linear(rosaq_ctx *ctx, const void *x, int M, int64_t ldx, const rosaq_rotation *r,
                  const rosaq_weight *w, void *y, int64_t ldy, void *stream);
