@@ -17,9 +17,10 @@
 // groups -- the first piece of its range: it stores that partial tile (fp32) in its own slot of a workspace
 // and raises its flag -- then whole tiles, and at the end of its range possibly a tile without its last groups:
 // it owns that tile, waits for the flags of the pairs that hold the rest (they went through it at the
-// start of their ranges, long before), adds their partial tiles in ascending K order and writes y.  Flags
-// hold the number of the launch, so nothing has to be reset.  The launch is cooperative: every pair is
-// resident, and a pair only ever waits for work that other pairs do first in their ranges.
+// start of their ranges, long before), adds their partial tiles in ascending K order and writes y.  A flag
+// has one writer and one reader, which puts it back to zero once the partial tile is in its shared memory:
+// every launch, replays of a captured launch included, starts from zero flags.  The launch is cooperative:
+// every pair is resident, and a pair only ever waits for work that other pairs do first in their ranges.
 //
 // Per CTA: warp 0 = weight-tile producer (bulk copies; one sub-ring of slots per dequantisation team),
 // 1 = activation producer (TMA, bytes of both CTAs counted on the leader's barrier), 2 = MMA issuer (leader
@@ -61,8 +62,7 @@ struct alignas(64) PfParams {
   int n_col_pairs, n_tok_blocks, M;
   int units;                  // (column pairs x token blocks) x groups
   float *partials;            // [pair][rank][256 tokens][128 columns]
-  unsigned *flags;            // [pair][rank]: the launch whose partial tile the slot holds
-  unsigned epoch;
+  unsigned *flags;            // [pair][rank]: 1 while the slot holds a partial tile that nobody has fetched yet
   int *status;
   long long wait_limit;
 };
@@ -355,7 +355,7 @@ linear_prefill_kernel(const __grid_constant__ PfParams p) {
         pf_epi_vote(true);
         if (lead) {
           __threadfence();
-          atomicExch(p.flags + 2 * pair + (int)rank, p.epoch);
+          atomicExch(p.flags + 2 * pair + (int)rank, 1u);
         }
         continue;
       }
@@ -372,7 +372,7 @@ linear_prefill_kernel(const __grid_constant__ PfParams p) {
             const unsigned *f = p.flags + 2 * h + (int)rank;
             got = false;
             for (long long it = 0; it < ab.limit && !got; ++it) {
-              got = pf_ld_acquire(f) == p.epoch;
+              got = pf_ld_acquire(f) != 0u;
               if (!got && (it & 15) == 15) {
                 if (ab.set()) break;
                 __nanosleep(64);
@@ -397,6 +397,7 @@ linear_prefill_kernel(const __grid_constant__ PfParams p) {
         }
         const bool landed = ab.wait_local(bar_merge, merge_phase);
         merge_phase ^= 1u;
+        if (lead && landed) p.flags[2 * h + (int)rank] = 0u;    // fetched: the slot is free for the next launch
         if (!pf_epi_vote(landed && !ab.set())) {
           alive = false;
           break;
@@ -579,7 +580,6 @@ int launch_linear_prefill(rosaq_ctx *ctx, const __half *x, int M, long long ldx,
   if (ctx->pl_partial_bytes < (size_t)n_pairs * 2 * kPfTokens * kTileN * sizeof(float)) return ROSAQ_ERR_ALLOC;
   p.partials = ctx->pl_partials;
   p.flags = ctx->pf_flags;
-  p.epoch = ++ctx->pf_epoch;
   p.status = ctx->d_status;
   p.wait_limit = ctx->wait_limit;
   return t.bits == 4 ? prefill_launch(linear_prefill_kernel<4>, p, n_pairs, s)

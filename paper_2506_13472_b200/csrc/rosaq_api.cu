@@ -154,7 +154,6 @@ int rosaq_create(rosaq_ctx **out, int device) {
   ctx->pl_sync = nullptr;
   ctx->pf_pairs = 0;
   ctx->pf_flags = nullptr;
-  ctx->pf_epoch = 0;
   st = cuda_status(cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 2 * sizeof(int)));   // [1]: scratch flag of argument checks
   if (st == ROSAQ_OK) st = cuda_status(cudaMemset(ctx->d_status, 0, 2 * sizeof(int)));
   // the stream-K workspace is taken here, once, so that no linear call ever allocates for it
@@ -222,6 +221,8 @@ int rosaq_last_status(rosaq_ctx *ctx, void *stream) {
     st = cuda_status(cudaMemset(ctx->sk_arrive, 0, rosaq::kSkCounterInts * sizeof(int)));
     if (st != ROSAQ_OK) return st;
     st = cuda_status(cudaMemset(ctx->pl_sync, 0, rosaq::kPlSyncWords * sizeof(unsigned)));
+    if (st != ROSAQ_OK) return st;
+    st = cuda_status(cudaMemset(ctx->pf_flags, 0, (size_t)ctx->sm_count * sizeof(unsigned)));
     if (st != ROSAQ_OK) return st;
   }
   return host;

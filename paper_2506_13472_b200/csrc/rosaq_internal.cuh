@@ -261,8 +261,7 @@ struct rosaq_ctx {
   std::vector<rosaq::PlanSchedule *> pl_schedules;   // one per geometry seen, owned
   // prefill tiles (pairs of CTAs; the partial tiles of a launch live in pl_partials)
   int pf_pairs;                                  // pairs the device keeps resident at once (0 until first asked for)
-  unsigned *pf_flags;                            // [pair][rank]: number of the launch whose partial tile is stored
-  unsigned pf_epoch;                             // number of the last launch
+  unsigned *pf_flags;                            // [pair][rank]: a partial tile is stored and not yet fetched; zero between launches
 };
 
 struct rosaq_weight {

@@ -189,6 +189,38 @@ def test_linear_prefill_tiles(ctx, M, d_in, d_out, k_salient, bits):
     w.free()
 
 
+def test_linear_prefill_tiles_replayed_from_a_graph_follow_their_input(ctx):
+    """A captured launch of the prefill tiles is replayed on other activations: the partial tiles that pairs of
+    CTAs exchange, and the flags that announce them, must be those of the replay, not of an earlier one."""
+    M, d_in, d_out = 520, 1024, 1152
+    W = synth.weights(d_in, d_out, seed=58, key="pfg", outlier_frac=0.01)
+    w = ctx.quantize(dev(W), None, bits=4, k_salient=128)
+    rng = synth.rng_for(58, "xg", M, d_in)
+    xa, xb = (rng.standard_normal((M, d_in)).astype(np.float16) for _ in range(2))
+    x, y = dev(xa), torch.empty((M, d_out), dtype=torch.float16, device="cuda")
+    ctx.set_linear_impl(5)
+    try:
+        want_a, want_b = (ctx.linear(dev(v), w, None).cpu().numpy() for v in (xa, xb))
+        ctx.linear(x, w, None, out=y)                       # warm-up outside the capture
+        torch.cuda.synchronize()
+        s = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                ctx.linear(x, w, None, out=y)
+        for v, want in ((xa, want_a), (xb, want_b), (xa, want_a)):
+            x.copy_(dev(v))
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            assert np.array_equal(y.cpu().numpy().view(np.uint16), want.view(np.uint16))
+        check_status(ctx)
+    finally:
+        ctx.set_linear_impl(0)
+    assert not np.array_equal(want_a, want_b)
+    w.free()
+
+
 def test_linear_strided_activations_and_output(ctx):
     c = H.config_tiny()
     w = ctx.quantize(dev(c["W"]), dev(c["R32"]), bits=4, k_salient=128)
