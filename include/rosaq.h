@@ -279,7 +279,7 @@ int rosaq_plan_free(rosaq_plan *plan);
 
 /* Test and tuning hook: the relative cost of an fp16 group, a quantized group and a started tile that
  * rosaq_plan_create (and the single calls, which plan internally) use from now on to cut a phase into
- * equal shares (defaults 10, 7, 1 for single CTAs and 15, 4, 1 for pairs; 1 <= cost <= 1000, tile >= 0).
+ * equal shares (defaults 12, 7, 1 for single CTAs and 10, 7, 1 for pairs; 1 <= cost <= 1000, tile >= 0).
  * Changes how K is divided among the CTAs, hence the fp32 summation order of later plans; plans already created keep theirs. */
 int rosaq_set_plan_costs(rosaq_ctx *ctx, int fp16_group, int quant_group, int tile);
 
@@ -298,7 +298,9 @@ int rosaq_plan_ctas(rosaq_ctx *ctx);
  * tile fp16; x_from[i] as in rosaq_op; copies[i] >= 1 (NULL: all 1) computes every tile of the operation that
  * many times, each copy writing an equal share of the token rows (what the library does, four-fold, for
  * block-diagonal rotations with a column permutation, whose output is a scatter bound by the store rate
- * of one SM).  An operation runs in the phase after the one it reads from; inside
+ * of one SM).  An operation runs in a later phase than the one it reads from; operations that neither read
+ * nor feed another one run in a phase of their own between the producers and their readers (the readers
+ * then find the producers' outputs complete instead of waiting for the exchange of shared tiles); inside
  * a phase the (operation, tile, group) list is cut into n_ctas contiguous ranges of equal cost, and a
  * range is a sequence of pieces (the groups of one tile).  Writes piece_begin[0..n_ctas] (CTA c owns pieces
  * piece_begin[c] .. piece_begin[c + 1] - 1, in the order it processes them) and, for the first max_pieces

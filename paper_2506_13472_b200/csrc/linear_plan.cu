@@ -162,18 +162,30 @@ __device__ __forceinline__ void epi_finish(uint32_t d_addr, bool both, int c_beg
     float acc[CH];
     epi_load_acc<CH>(d_addr, both, c0, acc);
     if (keep) {
-      for (int i = 1; i < S; ++i) {
+      // two holders' tiles per round trip to L2 (a round trip costs 1.4 us and more while the weight stream
+      // runs, and the readers of this tile wait for it), added in holder order
+      for (int i = 1; i < S; i += 2) {
         const float *src = src0 + (long long)i * slot_floats + c0 * kTileN;
-        float w[CH];
+        const bool two = i + 1 < S;
+        const float *src2 = two ? src + slot_floats : src;
+        float w[CH], w2[CH];
         if (c0 + CH <= M) {
 #pragma unroll
           for (int e = 0; e < CH; ++e) w[e] = __ldcg(src + e * kTileN);
+#pragma unroll
+          for (int e = 0; e < CH; ++e) w2[e] = __ldcg(src2 + e * kTileN);
         } else {
 #pragma unroll
           for (int e = 0; e < CH; ++e) w[e] = c0 + e < M ? __ldcg(src + e * kTileN) : 0.f;
+#pragma unroll
+          for (int e = 0; e < CH; ++e) w2[e] = c0 + e < M ? __ldcg(src2 + e * kTileN) : 0.f;
         }
 #pragma unroll
         for (int e = 0; e < CH; ++e) acc[e] = __fadd_rn(acc[e], w[e]);
+        if (two) {
+#pragma unroll
+          for (int e = 0; e < CH; ++e) acc[e] = __fadd_rn(acc[e], w2[e]);
+        }
       }
     }
     __half *yp = y_col + (long long)c0 * ldy;
@@ -721,7 +733,20 @@ int plan_build_schedule(const std::vector<PlanGeom> &ops, int n_ctas, const int 
     if (ops[i].n_tiles < 1 || ops[i].groups < 1 || ops[i].g_fp16 < 0 || ops[i].g_fp16 > ops[i].groups) return ROSAQ_ERR_INVALID_ARG;
     if (ops[i].rep < 1 || ops[i].rep > 16) return ROSAQ_ERR_INVALID_ARG;
     if (ops[i].dep >= i) return ROSAQ_ERR_INVALID_ARG;
-    phase[i] = ops[i].dep < 0 ? 0 : phase[ops[i].dep] + 1;
+  }
+  // Phases: an operation runs after the one whose output it reads.  Operations that neither read nor feed
+  // another one go BETWEEN the producers and their consumers: while the CTAs work through them, the
+  // epilogue warps close the producers' shared tiles in the background (partial tiles through L2, counters:
+  // 6 to 9 us on a 7B layer), so that the consumers' activation copies find those outputs complete.
+  std::vector<char> feeds(n, 0);
+  bool any_dep = false, any_free = false;
+  for (int i = 0; i < n; ++i)
+    if (ops[i].dep >= 0) feeds[ops[i].dep] = 1, any_dep = true;
+  for (int i = 0; i < n; ++i) any_free = any_free || (ops[i].dep < 0 && !feeds[i]);
+  const int step = any_dep && any_free ? 2 : 1;
+  for (int i = 0; i < n; ++i) {
+    if (ops[i].dep >= 0) phase[i] = phase[ops[i].dep] + step;
+    else phase[i] = (step == 2 && !feeds[i]) ? 1 : 0;
     n_phases = std::max(n_phases, phase[i] + 1);
   }
   std::vector<std::vector<PlanSeg>> per_cta(n_ctas);

@@ -179,11 +179,11 @@ constexpr int kPlSyncWords = kPlSyncArrive + kPlMaxCounters;
 // Relative cost of the work items when a phase is cut into equal shares.  Both kinds of group cost the
 // tensor pipe eight MMAs (about 700 cycles in place); an fp16 group also moves 32 KB, which takes an SM's
 // share of the HBM bandwidth about 1400 cycles when every SM streams fp16 tiles, less when some run
-// quantized groups next to it.  Measured on the 7B decoder layer: 10 : 7 is best (10 : 3 ... 10 : 10 all
-// within 10 %).  Every tile a CTA starts costs a little for switching accumulators; a tile copy whose
+// quantized groups next to it.  Measured on the 7B decoder layer: 12 : 7 (64.7 us per step; 10 : 7 65.4,
+// 14 : 7 64.9, 10 : 5 65.6; 10 : 3 ... 10 : 10 all within 10 %).  Every tile a CTA starts costs a little for switching accumulators; a tile copy whose
 // output is scattered keeps the epilogue warps busy for about as long as seven quantized groups keep
 // the MMA threads.
-constexpr int kPlanCostFp16 = 10, kPlanCostQuant = 7, kPlanCostTile = 1, kPlanCostScatterTile = 48;
+constexpr int kPlanCostFp16 = 12, kPlanCostQuant = 7, kPlanCostTile = 1, kPlanCostScatterTile = 48;
 // Pairs of CTAs: a quantized group costs each SM half the MMAs, but the measured layer step is again
 // shortest near 10 : 7 (76 us; 85 us at 12 : 4, 90 us at 15 : 4) -- a pair is not bound by its bytes either.
 constexpr int kPlanPairCostFp16 = 10, kPlanPairCostQuant = 7, kPlanPairCostTile = 1, kPlanPairCostScatterTile = 64;

@@ -1,6 +1,7 @@
 """Host logic of the persistent multi-operation launch (no GPU): how rosaq_plan divides a list of
 operations among the CTAs of its grid.  Checked here: every (operation, tile, group) is held exactly once;
-an operation that reads another's output is processed after it by every CTA; the holders of a shared tile
+an operation that reads another's output is processed after it by every CTA, with the operations that
+depend on nothing and feed nothing in between; the holders of a shared tile
 are consecutive in K, own consecutive partial-tile slots and one counter; at least one holder closes the
 tile, the closers are exactly the holders whose range ends in the tile, and they split the token rows;
 the shares of a phase are equal up to one work item."""
@@ -10,7 +11,7 @@ import pytest
 
 from paper_2506_13472_b200 import binding as rb
 
-COST_FP16, COST_QUANT, COST_TILE, COST_SCATTER_TILE = 10, 7, 1, 48
+COST_FP16, COST_QUANT, COST_TILE, COST_SCATTER_TILE = 12, 7, 1, 48
 
 LAYER_7B = dict(  # rot(attn), rot(mlp), rot(o) head-wise, down, q, k, v, o, gate, up
     n_tiles=[32, 32, 32, 32, 32, 32, 32, 32, 86, 86], groups=[32, 32, 1, 86, 32, 32, 32, 32, 32, 32],
@@ -23,15 +24,21 @@ CASES = {
     "tiny": (dict(n_tiles=[4, 2], groups=[4, 4], g_fp16=[4, 1], x_from=[-1, 0]), 148),     # fewer items than CTAs
     "13b-gateup": (dict(n_tiles=[40, 108, 108], groups=[40] * 3, g_fp16=[40, 1, 1], x_from=[-1, 0, 0]), 148),
     "chain": (dict(n_tiles=[3, 5, 2], groups=[7, 3, 5], g_fp16=[0, 3, 1], x_from=[-1, 0, 1]), 5),
+    "filler": (dict(n_tiles=[3, 4, 2], groups=[5, 6, 5], g_fp16=[5, 1, 1], x_from=[-1, -1, 0]), 6),   # op 1 feeds nobody
     "one-cta": (dict(n_tiles=[3, 2], groups=[2, 2], g_fp16=[1, 0], x_from=[-1, -1]), 1),
     "copies": (dict(n_tiles=[5, 3], groups=[3, 4], g_fp16=[3, 1], x_from=[-1, 0], copies=[3, 1]), 7),
 }
 
 
 def phases(x_from):
+    """An operation runs after the one it reads from; operations that neither read nor feed another one are
+    placed between the producers and their consumers (they fill the time the producers' exchange takes)."""
+    feeds = {f for f in x_from if f >= 0}
+    free = [i for i, f in enumerate(x_from) if f < 0 and i not in feeds]
+    step = 2 if feeds and free else 1
     ph = []
     for i, f in enumerate(x_from):
-        ph.append(0 if f < 0 else ph[f] + 1)
+        ph.append(ph[f] + step if f >= 0 else (1 if step == 2 and i in free else 0))
     return ph
 
 
