@@ -1,10 +1,11 @@
 // The GEMM stage  y = x . W^  (Eq. 3) for prefill-sized batches: more than 128 tokens.
 //
 // Why another kernel.  With a few hundred tokens the stage is bound by the tensor pipe, not by the weight
-// stream, and what counts is the width of an MMA and how often an operand byte is fetched from L2: a
-// tcgen05.mma of 128 x N x 16 runs at full rate only from N = 256 on (128 cycles; 64 cycles for N = 128 is half
-// rate), and a CTA that multiplies 128 columns with 256 tokens on its own pulls 64 KB of activations per
-// 128-channel group.  Here two CTAs of a cluster (adjacent SMs) share a 256-column x 256-token tile as a
+// stream, and what counts is how many tokens share one dequantisation of a weight tile and how often an
+// operand byte is fetched from L2: a tcgen05.mma of 128 x N x 16 runs at full rate from N = 128 on (64
+// cycles, 128 for N = 256; 55 for N = 64 is 58 %), a weight tile dequantised for 128 tokens costs as many
+// instructions as one dequantised for 256, and a CTA that multiplies 128 columns with 256 tokens on its own
+// pulls 64 KB of activations per 128-channel group.  Here two CTAs of a cluster (adjacent SMs) share a 256-column x 256-token tile as a
 // cta_group::2 pair: rank r dequantises column tile 2 c + r into its own tensor memory (the A operand, 128
 // lanes each) and loads 128 of the 256 token rows (its half of the B operand, 32 KB per group), the leader
 // issues M = 256, N = 256 MMAs for both, and each CTA ends up with the accumulator of its own 128 columns for
