@@ -73,6 +73,7 @@ struct PlProblem {
   int dep;                    // problem whose output this one reads, or -1
   unsigned dep_target;        // finishing events that complete problem `dep`
   int signal;                 // some problem reads this one's output: count finishing events
+  int m;                      // token rows of this problem (<= the launch's token capacity)
 };
 
 struct alignas(64) PlParams {
@@ -227,9 +228,14 @@ __device__ __forceinline__ void epi_store_partial(uint32_t d_addr, bool both, in
 // 222 cycles of each SM's tensor pipe per 128-channel group where a single CTA needs 440 -- less than the
 // 375 cycles the group's bytes take.  Barriers that both CTAs feed live in the leader; its commits are
 // multicast to both.
-template <int kBits, bool kPair>
+// kMode 2: a single CTA with accumulators of 128 tokens: two of them (one per piece parity) and the four
+// operand buffers fill the tensor memory, so there is one issuing thread, as in a pair; a group then costs
+// eight MMAs of N = 128 (64 cycles each: the full rate of the pipe) and its dequantisation serves twice the tokens.
+template <int kBits, int kMode>
 __global__ void __launch_bounds__(kPlThreads, 1)
 linear_plan_kernel(const __grid_constant__ PlParams p) {
+  constexpr bool kPair = kMode == 1, kBig = kMode == 2, kOne = kMode != 0;
+  constexpr int kTok = kBig ? 2 * kPlTokens : kPlTokens;       // token capacity of an accumulator
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int MT = p.MT;
@@ -272,7 +278,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       mbar_init(bar_s_empty + 8 * i, 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_d_full + 8 * i, kPair ? 1 : 2);            // the issuing threads
+      mbar_init(bar_d_full + 8 * i, kOne ? 1 : 2);             // the issuing threads
       mbar_init(bar_d_empty + 8 * i, (kPair ? 2 : 1) * (kPlEpiThreads / 32));   // one arrival per epilogue warp
       mbar_init(bar_drain + 8 * i, 1);
     }
@@ -293,7 +299,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
   }
   tc_fence_after();
   const uint32_t tmem = misc_ptr[0];
-  const uint32_t a_col0 = (kPair ? 2 : 4) * kPlTokens;         // operand buffers follow the accumulators
+  const uint32_t a_col0 = (kPair ? 2 : 4) * kPlTokens;         // operand buffers follow the accumulators (two of 128 columns when kBig)
   const int qbytes = quant_tile_bytes(kBits);
 
   if (warp == 0) {
@@ -408,9 +414,9 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
     // j mod 2 == i (operand buffers i and i + 2) and accumulates them into its own tile; per group one
     // wait, eight MMAs, one commit.  Every piece is committed by both (an issuer without a group in a
     // one-group piece arrives by hand), so the epilogue waits for one barrier.
-    if (lane == 0 && is_lead && !(kPair && warp == 3)) {       // (a pair has one issuing thread)
+    if (lane == 0 && is_lead && !(kOne && warp == 3)) {        // (a pair, or a CTA with wide accumulators, has one issuing thread)
       const int me = warp - 2;
-      constexpr int kStep = kPair ? 1 : 2;                     // issuers that share the stream
+      constexpr int kStep = kOne ? 1 : 2;                      // issuers that share the stream
       // M = 128 output columns (256 for a pair), N = MT tokens
       const uint32_t idesc = (1u << 4) | ((uint32_t)(MT >> 3) << 17) | ((kPair ? 16u : 8u) << 24);
       const uint64_t desc0 = make_b_desc(x_ring);
@@ -422,9 +428,9 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         const int buf = nseg & 1;
         if (!ab.wait(bar_d_empty + 8 * buf, ((nseg >> 1) & 1) ^ 1u)) break;   // the piece before last has been drained
         tc_fence_after();
-        const uint32_t d_tmem = tmem + (uint32_t)(kPair ? buf : 2 * buf + me) * kPlTokens;
+        const uint32_t d_tmem = tmem + (uint32_t)(kOne ? buf : 2 * buf + me) * kTok;
         uint32_t accumulate = 0;
-        const int g_first = kPair ? s.g_begin : s.g_begin + ((me - j) & 1), j_base = j - s.g_begin;
+        const int g_first = kOne ? s.g_begin : s.g_begin + ((me - j) & 1), j_base = j - s.g_begin;
         j += s.g_end - s.g_begin;
         for (int g = g_first; g < s.g_end; g += kStep) {
           const int j = j_base + g;
@@ -528,14 +534,14 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       const PlProblem &P = p.prob[s.prob];
       const int buf = nseg & 1;
       // the piece's groups have positions j0 .. in the CTA's stream: even ones went to issuer 0's tile
-      const bool both = !kPair && s.g_end - s.g_begin > 1;
-      const int first_acc = (both || kPair) ? 0 : (j0 & 1);
+      const bool both = !kOne && s.g_end - s.g_begin > 1;
+      const int first_acc = (both || kOne) ? 0 : (j0 & 1);
       j0 += s.g_end - s.g_begin;
       bool have_d = ab.wait(bar_d_full + 8 * buf, (nseg >> 1) & 1);
       have_d = __all_sync(0xffffffffu, have_d && !ab.set());
       if (!have_d) break;
       tc_fence_after();
-      const uint32_t d_addr = lane_addr + (uint32_t)(kPair ? buf : 2 * buf + first_acc) * kPlTokens;
+      const uint32_t d_addr = lane_addr + (uint32_t)(kOne ? buf : 2 * buf + first_acc) * kTok;
       const int n_glob = (tile_mul * s.tile + (int)rank) * kTileN + n;
       const bool n_ok = n_glob < P.d_out;
       const long long out_col = n_ok ? (P.col_map ? P.col_map[n_glob] : n_glob) : 0;
@@ -556,9 +562,10 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         if (ab.set()) break;
       }
       if (sole || keep) {
-        const int t0 = s.tok_begin, t1 = s.tok_end < p.M ? s.tok_end : p.M;     // token rows this piece writes
-        if (wide) epi_finish<16>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, p.M, n_ok, t0, t1, y_out + out_col, ldy);
-        else epi_finish<8>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, p.M, n_ok, t0, t1, y_out + out_col, ldy);
+        // token rows this piece writes (the schedule counts them in 64ths of the capacity)
+        const int t0 = s.tok_begin * (kTok / kPlTokens), t1 = min(s.tok_end * (kTok / kPlTokens), P.m);
+        if (wide) epi_finish<16>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, P.m, n_ok, t0, t1, y_out + out_col, ldy);
+        else epi_finish<8>(d_addr, both, c_begin, c_end, keep, S, src0, slot_step, P.m, n_ok, t0, t1, y_out + out_col, ldy);
         tc_fence_before();
         __syncwarp();                                          // one arrival per warp, where the issuers wait
         if (lane == 0) {
@@ -578,8 +585,8 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
       // accumulator back, count this CTA in
       {
         float *dst = p.partials + ((long long)tile_mul * (s.slot0 + s.contrib_idx) + rank) * p.slot_floats + n;
-        if (wide) epi_store_partial<16>(d_addr, both, c_begin, c_end, p.M, dst);
-        else epi_store_partial<8>(d_addr, both, c_begin, c_end, p.M, dst);
+        if (wide) epi_store_partial<16>(d_addr, both, c_begin, c_end, P.m, dst);
+        else epi_store_partial<8>(d_addr, both, c_begin, c_end, P.m, dst);
       }
       tc_fence_before();
       __syncwarp();
@@ -602,7 +609,7 @@ linear_plan_kernel(const __grid_constant__ PlParams p) {
         // (the two warps of a quadrant take alternate batches of eight rows; 32 loads are in flight per
         // thread and round; a holder index past S adds +0, which changes nothing)
         const int nc = s.n_closers;
-        const int t0 = s.tok_begin, t1 = s.tok_end < p.M ? s.tok_end : p.M;
+        const int t0 = s.tok_begin * (kTok / kPlTokens), t1 = min(s.tok_end * (kTok / kPlTokens), P.m);
         for (int r0 = s.closer_idx + ((warp - kPlFirstEpiWarp) >> 2) * 8 * nc; r0 < t1; r0 += 16 * nc) {
           float acc[8];
 #pragma unroll
@@ -891,10 +898,12 @@ static int plan_launch_kernel(K kern, const PlanLaunch &l, const PlParams &q, si
 // not available.
 int plan_units(rosaq_ctx *ctx, bool pair) {
   if (ctx->pl_ctas <= 0) {
-    if (plan_set_attrs(linear_plan_kernel<4, false>, kPlSmemBytes) != ROSAQ_OK ||
-        plan_set_attrs(linear_plan_kernel<3, false>, kPlSmemBytes) != ROSAQ_OK ||
-        plan_set_attrs(linear_plan_kernel<4, true>, kPlSmemBytes) != ROSAQ_OK ||
-        plan_set_attrs(linear_plan_kernel<3, true>, kPlSmemBytes) != ROSAQ_OK)
+    if (plan_set_attrs(linear_plan_kernel<4, 0>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<3, 0>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<4, 1>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<3, 1>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<4, 2>, kPlSmemBytes) != ROSAQ_OK ||
+        plan_set_attrs(linear_plan_kernel<3, 2>, kPlSmemBytes) != ROSAQ_OK)
       return 0;
     int p = ctx->sm_count;
     if (p > kPlanMaxCtas) p = kPlanMaxCtas;
@@ -911,7 +920,7 @@ int plan_units(rosaq_ctx *ctx, bool pair) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, linear_plan_kernel<4, true>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, linear_plan_kernel<4, 1>, &cfg) != cudaSuccess) {
       (void)cudaGetLastError();
       clusters = 0;
     }
@@ -983,12 +992,13 @@ void plan_free_schedules(rosaq_ctx *ctx) {
 // Checks the ops, finds their schedule, makes sure the exchange workspace is large enough and fills the
 // kernel parameters.  May allocate (a new geometry, a larger workspace); launches nothing.
 int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *out) {
-  if (n < 1 || n > kPlanMaxOps || M < 1 || M > kPlTokens) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (n < 1 || n > kPlanMaxOps || M < 1 || M > 2 * kPlTokens) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
   std::vector<PlanGeom> geom(n);
   int bits = 0;
+  const bool big = M > kPlTokens;                      // accumulators of 128 tokens, single CTAs, one issuing thread
   // pairs of CTAs (two adjacent column tiles per MMA) unless an operand's adjacent tiles multiply different
   // channels (a block-diagonal operand with an odd number of groups per block) or pairs are switched off
-  bool pair = ctx->pl_mode != 1 && plan_units(ctx, true) > 0;
+  bool pair = !big && ctx->pl_mode != 1 && plan_units(ctx, true) > 0;
   for (int i = 0; i < n && pair; ++i) pair = ops[i].t->block_groups % 2 == 0;
   const int tile_div = pair ? 2 : 1;
   for (int i = 0; i < n; ++i) {
@@ -1041,7 +1051,8 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
     const TiledOperand &t = *ops[i].t;
     const __half *x = ops[i].dep >= 0 ? ops[ops[i].dep].y : ops[i].x;
     const long long ldx = ops[i].dep >= 0 ? ops[ops[i].dep].ldy : ops[i].ldx;
-    if (!plan_encode_x(&q->xmap[i], x, M, ldx, t.d_in, MTL)) {
+    const int m = ops[i].m > 0 ? ops[i].m : M;
+    if (m > M || !plan_encode_x(&q->xmap[i], x, m, ldx, t.d_in, MTL)) {
       delete q;
       return ROSAQ_ERR_CUDA;
     }
@@ -1058,6 +1069,7 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
     P.dep = ops[i].dep;
     P.dep_target = ops[i].dep >= 0 ? (unsigned)tile_div * s->done_target[ops[i].dep] : 0u;   // both CTAs of a pair count
     P.signal = 0;
+    P.m = m;
   }
   for (int i = 0; i < n; ++i)
     if (ops[i].dep >= 0) q->prob[ops[i].dep].signal = 1;
@@ -1075,6 +1087,7 @@ int plan_prepare(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, PlanLaunch *ou
   out->params = q;
   out->n_ctas = tile_div * s->n_ctas;
   out->pair = pair;
+  out->big = big;
   out->bits = bits == 3 ? 3 : 4;
   out->partial_bytes = need;
   return ROSAQ_OK;
@@ -1092,10 +1105,12 @@ int plan_launch(rosaq_ctx *ctx, const PlanLaunch &l, cudaStream_t s) {
   q->partials = ctx->pl_partials;                      // the workspace may have grown since the plan was made
   q->wait_limit = ctx->wait_limit;
   const size_t smem = plan_smem_bytes(l.pair ? q->MT / 2 : q->MT, q->NW, l.pair ? kPlPairStages : kPlStages);
-  if (l.pair) return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, true>, l, *q, smem, s)
-                                 : plan_launch_kernel(linear_plan_kernel<4, true>, l, *q, smem, s);
-  return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, false>, l, *q, smem, s)
-                     : plan_launch_kernel(linear_plan_kernel<4, false>, l, *q, smem, s);
+  if (l.pair) return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, 1>, l, *q, smem, s)
+                                 : plan_launch_kernel(linear_plan_kernel<4, 1>, l, *q, smem, s);
+  if (l.big) return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, 2>, l, *q, smem, s)
+                                : plan_launch_kernel(linear_plan_kernel<4, 2>, l, *q, smem, s);
+  return l.bits == 3 ? plan_launch_kernel(linear_plan_kernel<3, 0>, l, *q, smem, s)
+                     : plan_launch_kernel(linear_plan_kernel<4, 0>, l, *q, smem, s);
 }
 
 }  // namespace rosaq

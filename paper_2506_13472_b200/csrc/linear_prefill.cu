@@ -5,11 +5,11 @@
 // operand byte is fetched from L2: a tcgen05.mma of 128 x N x 16 runs at full rate from N = 128 on (64
 // cycles, 128 for N = 256; 55 for N = 64 is 58 %), a weight tile dequantised for 128 tokens costs as many
 // instructions as one dequantised for 256, and a CTA that multiplies 128 columns with 256 tokens on its own
-// pulls 64 KB of activations per 128-channel group.  Here two CTAs of a cluster (adjacent SMs) share a 256-column x 256-token tile as a
-// cta_group::2 pair: rank r dequantises column tile 2 c + r into its own tensor memory (the A operand, 128
-// lanes each) and loads 128 of the 256 token rows (its half of the B operand, 32 KB per group), the leader
-// issues M = 256, N = 256 MMAs for both, and each CTA ends up with the accumulator of its own 128 columns for
-// all 256 tokens.  A weight tile is dequantised once per 256 tokens.
+// pulls 64 KB of activations per 128-channel group.  Here two CTAs of a cluster (adjacent SMs) share a
+// 256-column x 256-token tile as a cta_group::2 pair: rank r dequantises column tile 2 c + r into its own
+// tensor memory (the A operand, 128 lanes each) and loads 128 of the 256 token rows (its half of the B
+// operand, 32 KB per group), the leader issues M = 256, N = 256 MMAs for both, and each CTA ends up with the
+// accumulator of its own 128 columns for all 256 tokens.  A weight tile is dequantised once per 256 tokens.
 //
 // Work is cut the stream-K way: the list of (tile, 128-channel group) units, token blocks of one column pair
 // next to each other so that the second one finds the packed weights in L2, is cut into one contiguous range

@@ -63,10 +63,28 @@ int ensure_workspace(rosaq_ctx *ctx, size_t bytes, cudaStream_t s) {
 }
 
 constexpr int kPrefillMinTiles = 40, kPrefillMinUnits = 36;
+constexpr int kBlockTokens = 128;
+
+int run_ops(rosaq_ctx *ctx, int M, int n, const PlanOp *ops, cudaStream_t s);
+
+// 65 ... 1536 tokens as blocks of 128: one operation of the persistent launch per block, all in one launch
+// (accumulators of 128 tokens; a weight tile is dequantised once per block).
+int run_token_blocks(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t, const int32_t *col_map,
+                     __half *y, long long ldy, cudaStream_t s) {
+  const int nb = (M + kBlockTokens - 1) / kBlockTokens;
+  if (nb > kPlanMaxOps) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  PlanOp ops[kPlanMaxOps];
+  for (int b = 0; b < nb; ++b) {
+    const int m = std::min(kBlockTokens, M - b * kBlockTokens);
+    ops[b] = PlanOp{x + (long long)b * kBlockTokens * ldx, ldx, -1, &t, col_map, y + (long long)b * kBlockTokens * ldy, ldy, m};
+  }
+  return run_ops(ctx, std::min(M, kBlockTokens), nb, ops, s);
+}
 
 int run_gemm(rosaq_ctx *ctx, const __half *x, int M, long long ldx, const TiledOperand &t, const int32_t *col_map,
              __half *y, long long ldy, cudaStream_t s) {
   if (ctx->impl == 1) return launch_linear_simt(ctx, x, M, ldx, t, col_map, y, ldy, s);
+  if (ctx->impl == 6 && M > 64 && M <= kBlockTokens * kPlanMaxOps) return run_token_blocks(ctx, x, M, ldx, t, col_map, y, ldy, s);
   // Large batches of tokens run a weight on 256-column x 256-token tiles shared by pairs of CTAs -- where
   // the launch is long enough to pay for the exchange of the tiles that two pairs share: at least
   // kPrefillMinTiles tiles and kPrefillMinUnits 128-channel groups per pair of SMs (measured against the
@@ -238,7 +256,7 @@ int64_t rosaq_set_wait_limit(rosaq_ctx *ctx, int64_t iterations) {
 int rosaq_set_linear_impl(rosaq_ctx *ctx, int impl) {
   if (!ctx) return 0;
   int prev = ctx->impl;
-  if (impl >= 0 && impl <= 5) ctx->impl = impl;
+  if (impl >= 0 && impl <= 6) ctx->impl = impl;
   return prev;
 }
 
@@ -553,7 +571,7 @@ int rosaq_plan_create(rosaq_ctx *ctx, int M, int n_ops, const rosaq_op *ops, ros
   if (!out) return ROSAQ_ERR_INVALID_ARG;
   *out = nullptr;
   if (!ctx || !ops || n_ops < 1 || M < 1) return ROSAQ_ERR_INVALID_ARG;
-  if (n_ops > kPlanMaxOps || M > 64) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
+  if (n_ops > kPlanMaxOps || M > 128) return ROSAQ_ERR_UNSUPPORTED_SHAPE;
   rosaq_plan *pl = new (std::nothrow) rosaq_plan();
   if (!pl) return ROSAQ_ERR_ALLOC;
   pl->M = M;

@@ -227,11 +227,13 @@ struct PlanOp {
   const int32_t *col_map;
   __half *y;
   long long ldy;
+  int m = 0;            // token rows of this op; 0: the plan's M
 };
 
 struct PlanLaunch {
   void *params = nullptr;   // kernel parameters (tensor maps, problem table), owned
   int n_ctas = 0, bits = 4;
+  bool big = false;         // accumulators of 128 tokens (more than 64 tokens per operation)
   bool pair = false;        // clusters of two CTAs sharing an MMA stream
   size_t partial_bytes = 0;
 };

@@ -152,7 +152,7 @@ def test_linear_headwise(ctx, bits, impl):
     run_linear_case(ctx, c["x"], c["W"], c["Rb32"], c["Rb16"], c["perm"], bits, 128, impl)
 
 
-@pytest.mark.parametrize("impl", [1, 0, 4, 5])
+@pytest.mark.parametrize("impl", [1, 0, 4, 5, 6])
 @pytest.mark.parametrize("M,d_in,d_out,bits,k_salient", [
     (1, 256, 8, 4, 128), (3, 256, 136, 3, 0), (17, 384, 128, 4, 384), (64, 1024, 640, 4, 128),
     (130, 512, 256, 3, 128), (257, 256, 200, 4, 0)])
@@ -187,6 +187,38 @@ def test_linear_prefill_tiles(ctx, M, d_in, d_out, k_salient, bits):
     assert np.array_equal(again.view(np.uint16), y.view(np.uint16))
     assert H.rel_fro(y, y0.astype(np.float64)) <= 2e-4
     w.free()
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("M", [65, 128, 200, 600])
+def test_linear_token_blocks_of_128(ctx, M, bits):
+    """More than 64 tokens as blocks of 128 in one persistent launch (implementation 6): accumulators of 128
+    tokens, a ragged last block, the dense rotation and the head-wise one with its column permutation (whose
+    tiles are computed four times over, each copy writing a quarter of the token rows) -- all against the
+    oracle, and the same bits on a second run."""
+    c = H.config_headwise()
+    d_in = c["W"].shape[0]
+    x = synth.rng_for(61, "xb", M, d_in).standard_normal((M, d_in)).astype(np.float16)
+    qd = H.oracle_quantized(c["W"], c["Rb32"], c["perm"], bits, 128)
+    w = ctx.quantize(dev(c["W"]), dev(c["Rb32"]), dev(c["perm"]), bits=bits, k_salient=128)
+    rot = ctx.rotation_create(dev(c["Rb16"]), dev(c["perm"]))
+    y_ref, xr_ref = orc.forward(x, qd, c["Rb16"], c["perm"], return_xrot=True)
+    ctx.set_linear_impl(6)
+    try:
+        xr = ctx.rotate(dev(x), rot)
+        y = ctx.linear(dev(x), w, rot).cpu().numpy()
+        again = ctx.linear(dev(x), w, rot).cpu().numpy()
+        check_status(ctx)
+    finally:
+        ctx.set_linear_impl(0)
+    assert H.rel_fro(xr.cpu().numpy(), xr_ref) <= 1e-3
+    assert H.rel_fro(y, y_ref) <= H.REL_TOL_Y
+    assert np.array_equal(again.view(np.uint16), y.view(np.uint16))
+    t = H.config_tiny()                                                       # a dense rotation too
+    xt = synth.rng_for(61, "xt", M, t["W"].shape[0]).standard_normal((M, t["W"].shape[0])).astype(np.float16)
+    run_linear_case(ctx, xt, t["W"], t["R32"], t["R16"], None, bits, 128, 6)
+    w.free()
+    rot.free()
 
 
 def test_linear_prefill_tiles_replayed_from_a_graph_follow_their_input(ctx):
@@ -422,7 +454,7 @@ def test_a_perm_that_is_not_a_permutation_is_a_status_code(ctx):
 
 # --------------------------------------------------------------------------- bounded waits
 @pytest.mark.parametrize("impl,d_in,d_out", [(3, 1024, 512), (0, 1024, 150 * 128), (4, 1024, 512), (4, 512, 512),
-                                               (5, 1024, 512)])
+                                               (5, 1024, 512), (6, 1024, 512)])
 def test_expired_waits_in_the_linear_kernels_leave_the_context_usable(ctx, impl, d_in, d_out):
     """With the wait limit cut to one poll the linear kernels (cluster split-K, equal shares with the
     workspace exchange, the persistent launch with and without a rotation) may give up anywhere: they must
@@ -431,7 +463,8 @@ def test_expired_waits_in_the_linear_kernels_leave_the_context_usable(ctx, impl,
     W = synth.weights(d_in, d_out, seed=91, key=f"tw{d_in}x{d_out}", outlier_frac=0.01)
     w = ctx.quantize(dev(W), None, bits=4, k_salient=128)
     rot = ctx.rotation_create(dev(H.config_tiny()["R16"])) if d_in == 512 else None
-    x = dev(synth.rng_for(91, "x", d_in).standard_normal((64, d_in)).astype(np.float16))
+    M = 96 if impl == 6 else 64                                # (implementation 6 is about more than 64 tokens)
+    x = dev(synth.rng_for(91, "x", d_in).standard_normal((M, d_in)).astype(np.float16))
     ctx.set_linear_impl(impl)
     try:
         want = ctx.linear(x, w, rot).cpu().numpy()

@@ -38,7 +38,7 @@ def householder_rotation(d, seed, key):
 
 
 @pytest.mark.parametrize("pairs", [True, False])
-@pytest.mark.parametrize("bits,M", [(4, 4), (3, 64), (4, 33), (3, 1)])
+@pytest.mark.parametrize("bits,M", [(4, 4), (3, 64), (4, 33), (3, 1), (4, 128), (3, 90)])
 def test_small_layer_plan_against_oracle_and_separate_calls(ctx, bits, M, pairs):
     """A decoder layer in miniature (d = 512, ffn = 1024, 4 heads): dense rotations for the attention and
     MLP inputs, a head-wise one with its permutation for the o_proj input, down_proj un-rotated."""
@@ -132,9 +132,9 @@ def test_plan_argument_errors(ctx):
         assert e.value.status == rb.ROSAQ_ERR_INVALID_ARG
     # column ranges of one wider buffer are distinct outputs
     ctx.plan_create(8, [(x, None, w4, wide[:, :128]), (xs, None, w4, wide[:, 128:])]).free()
-    x65 = torch.zeros((65, 256), dtype=torch.float16, device="cuda")
+    x129 = torch.zeros((129, 256), dtype=torch.float16, device="cuda")
     with pytest.raises(rb.RosaqError) as e:
-        ctx.plan_create(65, [(x65, None, w4, empty(65, 128))])
+        ctx.plan_create(129, [(x129, None, w4, empty(129, 128))])
     assert e.value.status == rb.ROSAQ_ERR_UNSUPPORTED_SHAPE
     assert ctx.last_status() == rb.ROSAQ_OK
 
